@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the decode / verify attention step over xTensor-mapped KV on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|verify|longctx|paged|tiny]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on a bounded sample (reported baseline)
+
+One step = one pass of the whole hot path over one batch: map pages for the tokens about to be written,
+append the new K/V rows, partition the work, split-KV attention, LSE combine, then roll the sequence
+length back so that every step sees the named context lengths.  Prints ONE JSON line (rank 0).
+
+Metric: KV tokens/s = sum of context lengths attended per step / step time; `value` is timed with CUDA
+events with all inputs resident in HBM, `e2e` through the same C-ABI calls with pinned HOST buffers for
+the step's inputs (q, new K/V rows) and output.  Consecutive steps rotate over independent copies of the
+batch so that no step finds its K/V in L2.  With N > 1 every rank runs the same workload on its own GPU
+(requests are independent: replicas, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2510_14686_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode_attention_kv_tokens_per_s"
+UNIT = "KV tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 << 20
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0]))
+                mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# reference arm: the oracle as it stands, on host cores, bounded sample per step
+# ------------------------------------------------------------------------------------------------------------
+def oracle_sample(name: str, max_requests: int):
+    batch = wl.make_batch(name, with_values=True, max_requests=max_requests)
+    return batch
+
+
+def time_oracle(batch, reps: int):
+    import oracle
+
+    qs, ks, vs = [r.q for r in batch.requests], [r.k for r in batch.requests], [r.v for r in batch.requests]
+    cores = min(os.cpu_count() or 1, len(qs))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.attention_batch(qs, ks, vs, batch.shape.scale, n_threads=cores)
+    dt = (time.perf_counter() - t0) / reps
+    return batch.kv_tokens / dt, dt, cores
+
+
+def sample_size(name: str) -> int:
+    return {"tiny": 4, "decode": 16, "verify": 8, "longctx": 1, "paged": 64}[name]
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    n = sample_size(args.workload)
+    batch = oracle_sample(args.workload, n)
+    _, dt1, _ = time_oracle(batch, 1)                      # doubles as warm-up; sizes the sample for a ~2 minute run
+    budget_s = 120.0
+    while dt1 * (args.steps + args.warmup) > budget_s and len(batch.requests) > 1:
+        keep = max(1, int(len(batch.requests) * budget_s / (dt1 * (args.steps + args.warmup))))
+        batch.requests = batch.requests[:keep]
+        _, dt1, _ = time_oracle(batch, 1)
+    for _ in range(args.warmup):
+        time_oracle(batch, 1)
+    tps, dt, cores = time_oracle(batch, max(1, args.steps))
+    s = batch.shape
+    sample = f"first {len(batch.requests)} of {s.batch} requests of '{args.workload}' ({batch.kv_tokens} KV tokens) per step"
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": workload_config(args.workload, s, world, note="CPU oracle on a bounded sample"),
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(name, s, world, note=None):
+    kv, ql = wl.draw_lengths(name)
+    cfg = {"workload": f"{name}: batch {s.batch}, {s.n_q_heads} q heads / {s.n_kv_heads} kv heads, head_dim {s.head_dim}, "
+                       f"q_len {sorted(set(int(x) for x in ql))}, context {int(kv.min())}..{int(kv.max())} (sum {int(kv.sum())}), seed {s.seed}",
+           "kv_tokens_per_step_per_gpu": int(kv.sum()), "kv_bytes_per_step_per_gpu": int(kv.sum()) * s.row_bytes,
+           "parallelism": f"replicas x{world} (requests are independent; no collective)",
+           "l2": "steps rotate over independent KV copies whose total size exceeds the 126 MB L2"}
+    if note:
+        cfg["note"] = note
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------------------
+class Replica:
+    """`copies` independent instances of the workload resident on one GPU, plus per-step inputs."""
+
+    def __init__(self, name: str, copies: int, device: int):
+        import torch
+
+        from paper_2510_14686_b200 import binding
+
+        self.torch, self.binding = torch, binding
+        self.name, self.s = name, wl.SHAPES[name]
+        s = self.s
+        self.kv, self.ql = wl.draw_lengths(name)
+        self.B = len(self.kv)
+        self.copies = copies
+        page = 2 << 20
+        pages = sum(-(-(-(-int(t) // 64) * 64 * s.row_bytes) // page) for t in self.kv) * copies + 4
+        self.ctx = binding.Context(s.n_q_heads, s.n_kv_heads, s.head_dim, self.B * copies, int(self.kv.max()) + 64,
+                                   pages * page, max_q_len=4, device=device)
+        gen = torch.Generator(device="cuda").manual_seed(s.seed)
+        self.slots = []
+        for c in range(copies):
+            row = []
+            for r in range(self.B):
+                sl = self.ctx.kv_reserve(expected_tokens=int(self.kv[r]))
+                pre = int(self.kv[r] - self.ql[r])            # cached before the step; the step appends q_len rows
+                self.ctx.kv_map_pages(sl, pre)
+                for t0 in range(0, pre, 1 << 15):
+                    n = min(pre - t0, 1 << 15)
+                    k = torch.randn((n, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+                    v = torch.randn((n, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+                    self.ctx.kv_append([sl], [n], k, v)
+                row.append(sl)
+            self.slots.append(np.array(row, np.int32))
+        rows = int(self.ql.sum())
+        self.rows = rows
+        self.q = torch.randn((rows, s.n_q_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+        self.k_new = torch.randn((rows, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+        self.v_new = torch.randn((rows, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+        self.out = torch.zeros_like(self.q)
+        # host side of the end-to-end path
+        self.h_q, self.h_k, self.h_v = (t.cpu().pin_memory() for t in (self.q, self.k_new, self.v_new))
+        self.h_out = torch.zeros_like(self.h_q).pin_memory()
+        self.d_q, self.d_k, self.d_v = torch.empty_like(self.q), torch.empty_like(self.k_new), torch.empty_like(self.v_new)
+        torch.cuda.synchronize()
+        self.pre = (self.kv - self.ql).astype(np.int64)
+        self.decode_only = bool((self.ql == 1).all())
+
+    def step(self, i: int, q=None, k_new=None, v_new=None):
+        ctx, slots = self.ctx, self.slots[i % self.copies]
+        q = self.q if q is None else q
+        ctx.kv_map_pages_many(slots, self.kv)                              # a1: pages for the tokens about to be written
+        ctx.kv_append(slots, self.ql, self.k_new if k_new is None else k_new, self.v_new if v_new is None else v_new)  # a2
+        if self.decode_only:                                               # a3 + a4 + a5
+            ctx.decode_attention(slots, q, self.out, None, self.s.scale)
+        else:
+            ctx.verify_attention(slots, self.ql, q, self.out, None, self.s.scale)
+        ctx.kv_set_len_many(slots, self.pre)                               # back to the named context lengths
+
+    def step_e2e(self, i: int):
+        t = self.torch
+        self.d_q.copy_(self.h_q, non_blocking=True)
+        self.d_k.copy_(self.h_k, non_blocking=True)
+        self.d_v.copy_(self.h_v, non_blocking=True)
+        self.step(i, self.d_q, self.d_k, self.d_v)
+        self.h_out.copy_(self.out, non_blocking=True)
+        t.cuda.current_stream().synchronize()                              # the caller reads the result every step
+
+
+def run_ours(args):
+    import torch
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        dist = None
+        torch.cuda.set_device(0)
+    dev = torch.cuda.current_device()
+    name = args.workload
+    s = wl.SHAPES[name]
+    kv, ql = wl.draw_lengths(name)
+    kv_bytes = int(kv.sum()) * s.row_bytes
+    copies = max(3, -(-3 * L2_BYTES // max(kv_bytes, 1))) if name != "longctx" else 2
+    copies = min(copies, 64)
+    rep = Replica(name, copies, dev)
+    tokens_per_step = int(kv.sum())
+    rows = int(ql.sum())
+    alg_bytes = kv_bytes + 2 * rows * s.n_q_heads * s.head_dim * 2
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(n_steps, fn, first=0):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for i in range(n_steps):
+            fn(first + i)
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for i in range(max(args.warmup, 3)):
+        rep.step(i)
+    rep.ctx.sync_check()
+
+    sampler = ClockSampler(dev)
+    if rank == 0:
+        sampler.start()
+    t_load0 = time.perf_counter()
+    st0 = rep.ctx.get_stats()
+    ms = timed(args.steps, rep.step)                                       # ---- the timed region ----
+    st1 = rep.ctx.get_stats()
+    launches = int(st1.kernel_launches - st0.kernel_launches)
+
+    # same steps again with per-kernel CUDA events (inside the library, on the launching stream)
+    rep.ctx.set_profiling(True)
+    p0 = rep.ctx.get_stats()
+    timed(args.steps, rep.step, first=args.steps)
+    p1 = rep.ctx.get_stats()
+    rep.ctx.set_profiling(False)
+    attn_ms = (p1.attn_kernel_ms - p0.attn_kernel_ms) / max(1, p1.attn_launches - p0.attn_launches)
+    comb_n = p1.combine_launches - p0.combine_launches
+    comb_ms = (p1.combine_kernel_ms - p0.combine_kernel_ms) / comb_n if comb_n else 0.0
+    app_ms = (p1.append_kernel_ms - p0.append_kernel_ms) / max(1, p1.append_launches - p0.append_launches)
+
+    for i in range(3):
+        rep.step_e2e(i)
+    ms_e2e = timed(args.steps, rep.step_e2e)
+
+    # keep the GPU under the same load until the clock sampler has seen it for a while
+    i = 0
+    while rank == 0 and time.perf_counter() - t_load0 < 1.5:
+        rep.step(i)
+        i += 1
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    rep.ctx.sync_check()
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    value = tokens_per_step * world * args.steps / (ms * 1e-3)
+    e2e_value = tokens_per_step * world * args.steps / (ms_e2e * 1e-3)
+    achieved = alg_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
+    h2d = int(rep.h_q.numel() + rep.h_k.numel() + rep.h_v.numel()) * 2
+    d2h = int(rep.h_out.numel()) * 2
+
+    # CPU baseline: the oracle, untouched, on this machine's host cores, on a bounded sample of the same workload
+    sample = oracle_sample(name, sample_size(name))
+    cpu_tps, cpu_dt, cores = time_oracle(sample, 1)
+
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(tpath) as f:
+            traffic = json.load(f).get(name)
+    except Exception:
+        pass
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": workload_config(name, s, world),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "attention_kernel (split-KV)",
+                     "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": attn_ms,
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "combine_kernel_ms": comb_ms, "append_kernel_ms": app_ms},
+        "cpu_baseline": {"value": cpu_tps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {len(sample.requests)} of {s.batch} requests ({sample.kv_tokens} KV tokens), 1 pass, {cpu_dt:.2f} s"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": launches, "clocks": clocks,
+        "hbm_gbs_whole_step": alg_bytes * world * args.steps / (ms * 1e-3) / 1e9,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=list(wl.SHAPES), default="decode")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

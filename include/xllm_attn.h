@@ -1,0 +1,224 @@
+/*
+ * xllm_attn.h -- C ABI of libxllm_attn.so
+ *
+ * Batched decode and speculative-verification grouped-query attention for NVIDIA B200 (sm_100a)
+ * over a per-request KV cache kept in an xTensor-style "logically contiguous, physically
+ * discrete" layout (xLLM technical report, section "Efficient Memory Management").
+ *
+ * Conventions for every call
+ *   - "host" / "device" says where a pointer must live.  Device pointers belong to the caller
+ *     (typically torch tensors); the library never frees them.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All
+ *     kernels are launched on it; no call synchronises the stream unless stated.
+ *   - Small host arrays (`slots`, `n_new`, `q_lens`) are consumed before the call returns.
+ *   - Every call returns an xllm_status; on failure the context state is unchanged and
+ *     xllm_last_error() describes the problem.  Nothing throws, aborts or traps.  All argument
+ *     and state checks run before any kernel is launched.  An asynchronous CUDA error or a device
+ *     side wait that gave up is reported by the next call (or xllm_sync_check) as XLLM_ERR_CUDA.
+ *   - A context is bound to one device and is not thread safe; callers serialise.
+ *   - bf16 tensors are raw 16-bit patterns; all tensors are dense and row major.
+ */
+#ifndef XLLM_ATTN_H
+#define XLLM_ATTN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xllm_ctx xllm_ctx; /* opaque: VA ranges, physical pages, page table, workspace */
+typedef int32_t xllm_status;
+
+#define XLLM_OK 0
+#define XLLM_ERR_INVALID (-1)     /* bad argument or call order (bad slot, q_len out of range, kv_len < q_len) */
+#define XLLM_ERR_OOM_PHYS (-2)    /* physical page pool exhausted (after reclaiming reusable pages) */
+#define XLLM_ERR_OOM_VA (-3)      /* no free slot / virtual address reservation failed */
+#define XLLM_ERR_NOT_MAPPED (-4)  /* the call would touch tokens beyond the slot's mapped pages */
+#define XLLM_ERR_CUDA (-5)        /* CUDA runtime / driver error, or a device-side bounded wait expired */
+#define XLLM_ERR_BUSY (-6)        /* slot still used by work in flight and XLLM_FLAG_NONBLOCKING_UNMAP set */
+#define XLLM_ERR_UNSUPPORTED (-7) /* head geometry not supported, or GPU work asked of a host-only context */
+
+/* xllm_config.flags */
+#define XLLM_FLAG_LAZY_PAGES 1u        /* create physical pages on first use instead of all at init */
+#define XLLM_FLAG_NONBLOCKING_UNMAP 2u /* unmapping a slot with work in flight returns BUSY instead of waiting */
+#define XLLM_FLAG_HOST_ONLY 4u         /* bookkeeping against an in-process fake of the driver: no GPU is touched, \
+                                          every kernel-launching call returns XLLM_ERR_UNSUPPORTED (host tests) */
+
+#define XLLM_TILE_TOKENS 64 /* tokens per KV tile block: unit of the private slot layout and of work splitting */
+#define XLLM_MAX_Q_LEN 8    /* upper bound accepted for xllm_config.max_q_len */
+
+typedef struct {
+    int32_t device;            /* CUDA device ordinal */
+    int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads */
+    int32_t n_kv_heads;        /* H_kv */
+    int32_t head_dim;          /* D: 64 or 128 */
+    int32_t max_slots;         /* number of request slots (virtual ranges) */
+    int32_t max_q_len;         /* largest q_len a verify call may carry, 1..XLLM_MAX_Q_LEN */
+    int64_t max_seq_len;       /* tokens of virtual range per slot ("MaxSeqLen") */
+    int64_t phys_budget_bytes; /* HBM budget for KV pages; the pool holds floor(budget / page_bytes) pages */
+    int64_t page_bytes;        /* 0 = the device's minimum VMM granularity; else a multiple of it */
+    uint32_t flags;
+    uint32_t fault_inject;     /* HOST_ONLY contexts: the fake driver fails its n-th page creation (0 = never) */
+} xllm_config;
+
+typedef struct {
+    int64_t page_bytes;
+    int64_t pages_total, pages_free, pages_allocated, pages_mapped, pages_reusable; /* by Status */
+    int64_t pages_mapped_total;   /* driver map operations so far (one per page) */
+    int64_t pages_unmapped_total; /* driver unmap operations so far */
+    int64_t pages_reused_total;   /* Reusable -> Mapped without a driver call */
+    double map_host_us;           /* host time spent inside driver map + set-access calls */
+    double unmap_host_us;         /* host time spent inside driver unmap calls */
+    int64_t tokens_appended;
+    int64_t attention_calls;
+    int64_t work_items;           /* attention work items launched in total */
+    int64_t partial_items;        /* of those, items that wrote a partial (split) result */
+    int64_t attn_launches;        /* attention kernel launches timed while profiling was on */
+    double attn_kernel_ms;        /* their summed device time (CUDA events on the caller's stream) */
+    double combine_kernel_ms;     /* same for the combine kernel */
+    double append_kernel_ms;      /* same for the append kernel */
+    int64_t combine_launches, append_launches;
+    int64_t kernel_launches;      /* kernels of this library launched so far (append, gather, attention, combine) */
+    int32_t sm_count;             /* CTAs of the persistent attention grid */
+    int32_t reserved;
+} xllm_stats;
+
+typedef struct {
+    uint64_t base;          /* device virtual address of the slot's range (0 before its first reserve) */
+    int64_t va_bytes;       /* size of the range */
+    int64_t kv_len;         /* tokens currently cached */
+    int64_t mapped_tokens;  /* tokens covered by the pages the live request owns */
+    int32_t pages_in_range; /* pages currently mapped in the range (owned + reusable tail) */
+    int32_t pages_owned;    /* of those, Status = Mapped */
+    int32_t live;           /* 1 between reserve and release */
+    int32_t row_bytes;      /* bytes per token: K and V of all KV heads, bf16 */
+} xllm_slot_info;
+
+/* One unit of attention work: a run of KV tile blocks of one (request, KV head, query rows) triple. */
+typedef struct {
+    int32_t req;         /* index into the call's request list */
+    int32_t kv_head;
+    int32_t tile_begin;  /* first tile block (XLLM_TILE_TOKENS tokens each) */
+    int32_t tile_end;    /* one past the last */
+    int16_t q_tok0;      /* first query token of the row group */
+    int16_t n_q_tok;     /* query tokens in the row group */
+    int16_t g0;          /* first query head inside the GQA group */
+    int16_t n_g;         /* query heads of the group covered; rows = n_q_tok * n_g <= 16 */
+    int32_t partial_idx; /* -1: the item covers the whole context and writes the final output;
+                            else index of its partial result in the split workspace */
+    int32_t unit;        /* id of the (request, KV head, row group) unit the item belongs to */
+} xllm_work_item;
+
+/* ---- life cycle ------------------------------------------------------------------------------- */
+
+/* Create a context: page pool of floor(phys_budget_bytes / page_bytes) pages (created now unless
+ * XLLM_FLAG_LAZY_PAGES), slot table, workspace.  (xTensor: pages are pre-allocated at service start.) */
+xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out);
+/* Synchronise the device, unmap and release every page and virtual range, free the workspace. */
+xllm_status xllm_shutdown(xllm_ctx *ctx);
+/* Message of the last failed call on this context (valid until the next call); ctx may be NULL for
+ * the message of a failed xllm_init. */
+const char *xllm_last_error(const xllm_ctx *ctx);
+/* Synchronise `cuda_stream` and report asynchronous failures (CUDA errors, expired device waits). */
+xllm_status xllm_sync_check(xllm_ctx *ctx, void *cuda_stream);
+
+/* ---- xTensor: virtual ranges and on-demand page mapping -------------------------------------------- */
+
+/* Give a new request a slot: one contiguous virtual range of max_seq_len tokens with no physical
+ * backing (xTensor, "each request is pre-allocated a logically contiguous virtual address space of
+ * MaxSeqLen").  max_seq_len must not exceed the context's.  A released slot whose pages were kept
+ * (Reusable) is preferred: the one whose page set fits `expected_tokens` best ("Physical Page Reuse");
+ * pass 0 when the size is unknown.  The first use of a slot id reserves its range with
+ * cuMemAddressReserve; the range is kept for later requests ("request ID reuse").  kv_len starts at 0. */
+xllm_status xllm_kv_reserve(xllm_ctx *ctx, int64_t max_seq_len, int64_t expected_tokens, int32_t *slot_out);
+
+/* Ensure the slot's live request owns pages covering at least min_tokens tokens ("On-demand Memory
+ * Mapping": free pages are mapped at the next contiguous position of the range).  Idempotent.  Pages
+ * come from the slot's own reusable tail first (no driver call), then the Free stack (cuMemMap +
+ * cuMemSetAccess), then reusable pages reclaimed from other slots.  Host-synchronous and not stream
+ * ordered: it returns with the mapping usable by kernels launched afterwards. */
+xllm_status xllm_kv_map_pages(xllm_ctx *ctx, int32_t slot, int64_t min_tokens);
+
+/* The same for n_req slots in one call (one scheduler step): slot slots[i] is grown to min_tokens[i].  Stops at
+ * the first failure; slots before it keep their new pages. */
+xllm_status xllm_kv_map_pages_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens);
+
+/* End a request.  mode 0: keep the pages mapped in the range, Status = Reusable, for the next request
+ * that takes the slot over; mode 1: unmap them back to the Free stack (waits for work in flight on the
+ * slot, or returns BUSY with XLLM_FLAG_NONBLOCKING_UNMAP).  kv_len becomes 0; the range stays reserved. */
+xllm_status xllm_kv_release(xllm_ctx *ctx, int32_t slot, int32_t mode);
+
+/* Set the number of cached tokens (0 <= kv_len <= mapped tokens): roll back rejected draft tokens. */
+xllm_status xllm_kv_set_len(xllm_ctx *ctx, int32_t slot, int64_t kv_len);
+
+/* The same for n_req slots in one call; all arguments are checked before any length changes. */
+xllm_status xllm_kv_set_len_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *kv_lens);
+
+xllm_status xllm_kv_slot_info(const xllm_ctx *ctx, int32_t slot, xllm_slot_info *info);
+
+/* Page table lookup for a byte offset inside a slot's range (xTensor Eq. 2): position of the page in the
+ * range, its PageID in the pool and the offset inside the page.  NOT_MAPPED if no page backs the offset. */
+xllm_status xllm_kv_page_of(const xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int32_t *page_pos,
+                            int32_t *page_id, int64_t *in_page_offset);
+
+/* Inspection (synchronous, for tests and tools): copy bytes to host memory, either through the slot's
+ * virtual range or through a temporary second mapping of one physical page. */
+xllm_status xllm_debug_read_slot(xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int64_t nbytes, void *host_dst);
+xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_offset, int64_t nbytes, void *host_dst);
+
+/* ---- KV writes ("write_kvcache": only a start address and offsets, no block table) ---------------------- */
+
+/* Append n_new[i] tokens to slot slots[i] for i < n_req: rows k_new / v_new (device, bf16,
+ * [sum n_new, H_kv, D], request-major) are written at token positions kv_len .. kv_len + n_new - 1 of each
+ * range and kv_len advances.  The target tokens must already be mapped (else NOT_MAPPED, nothing written).
+ * A slot may appear once per call. */
+xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new,
+                           const void *k_new, const void *v_new, void *cuda_stream);
+
+/* Copy tokens first_token .. first_token + n_tokens - 1 of a slot back out as dense rows
+ * (device, bf16, [n_tokens, H_kv, D] each): the inverse of append, for tests and KV migration. */
+xllm_status xllm_kv_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int64_t n_tokens, void *k_out,
+                           void *v_out, void *cuda_stream);
+
+/* ---- attention ----------------------------------------------------------------------------------------- */
+
+/* Decode: one query token per request.  q, out: device bf16 [n_req, H_q, D]; lse_out: device fp32
+ * [n_req, H_q] (natural log) or NULL.  Request i attends to all kv_len tokens of slots[i]
+ * (softmax(scale * q k^T) v per query head, head h using KV head h / (H_q / H_kv)).  Same as
+ * xllm_verify_attention with every q_len = 1. */
+xllm_status xllm_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const void *q, void *out,
+                                  float *lse_out, float scale, void *cuda_stream);
+
+/* Speculative verification (m draft tokens + 1: "m+1 Q matrices against the same K"): request i carries
+ * q_lens[i] query tokens (1..max_q_len), the newest q_lens[i] tokens of its slot, already appended.  Query
+ * token t of request i sits at position kv_len - q_lens[i] + t and sees keys 0 .. that position (causal
+ * among the drafts, full view of the older context).  q, out: device bf16 [sum q_lens, H_q, D],
+ * request-major; lse_out: device fp32 [sum q_lens, H_q] or NULL.  Requires kv_len >= q_len.
+ * One launch of the split-KV kernel (each K/V byte read once for all query rows of a GQA group) and,
+ * when a sequence was split across CTAs, one launch of the log-sum-exp combine kernel. */
+xllm_status xllm_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
+                                  const void *q, void *out, float *lse_out, float scale, void *cuda_stream);
+
+/* ---- work partition (host only; exposed so that it can be checked without a GPU) ---------------------------- */
+
+/* Split the step's KV tile blocks into per-CTA runs of near-equal cost (hierarchical DP load balance,
+ * layer 3: equalise tokens per compute unit, split long sequences).  kv_lens / q_lens: host [n_req].
+ * Writes at most max_items items, grouped by CTA: CTA c owns items cta_begin[c] .. cta_begin[c+1]-1
+ * (cta_begin has n_ctas + 1 entries).  Returns INVALID if max_items is too small or a size is bad. */
+xllm_status xllm_plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
+                                int32_t n_kv_heads, int32_t n_ctas, xllm_work_item *items, int32_t max_items,
+                                int32_t *cta_begin, int32_t *n_items_out, int32_t *n_units_out,
+                                int32_t *n_partials_out);
+
+/* ---- statistics ------------------------------------------------------------------------------------------ */
+
+xllm_status xllm_get_stats(const xllm_ctx *ctx, xllm_stats *stats);
+/* When on, each kernel launch is bracketed by CUDA events on the caller's stream and its device time
+ * is accumulated into xllm_stats (read after synchronising the stream; xllm_get_stats resolves them). */
+xllm_status xllm_set_profiling(xllm_ctx *ctx, int32_t on);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XLLM_ATTN_H */

@@ -1,0 +1,257 @@
+"""ctypes binding of ``libxllm_attn.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs inside the shared library; this module converts Python values to C
+arguments and turns negative status codes into :class:`XllmError`.  There is no Python or CPU
+fallback: if the library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libxllm_attn.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2510_14686_b200.build` "
+        "(nvcc, sm_100a). There is no CPU fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK, ERR_INVALID, ERR_OOM_PHYS, ERR_OOM_VA, ERR_NOT_MAPPED, ERR_CUDA, ERR_BUSY, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7
+FLAG_LAZY_PAGES, FLAG_NONBLOCKING_UNMAP, FLAG_HOST_ONLY = 1, 2, 4
+TILE_TOKENS = 64
+STATUS_NAMES = {0: "OK", -1: "INVALID", -2: "OOM_PHYS", -3: "OOM_VA", -4: "NOT_MAPPED", -5: "CUDA", -6: "BUSY",
+                -7: "UNSUPPORTED"}
+
+
+class XllmError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"xllm status {status} ({STATUS_NAMES.get(status, '?')}): {message}")
+        self.status = status
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("device", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("max_slots", ctypes.c_int32), ("max_q_len", ctypes.c_int32),
+                ("max_seq_len", ctypes.c_int64), ("phys_budget_bytes", ctypes.c_int64), ("page_bytes", ctypes.c_int64),
+                ("flags", ctypes.c_uint32), ("fault_inject", ctypes.c_uint32)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("page_bytes", ctypes.c_int64), ("pages_total", ctypes.c_int64), ("pages_free", ctypes.c_int64),
+                ("pages_allocated", ctypes.c_int64), ("pages_mapped", ctypes.c_int64), ("pages_reusable", ctypes.c_int64),
+                ("pages_mapped_total", ctypes.c_int64), ("pages_unmapped_total", ctypes.c_int64),
+                ("pages_reused_total", ctypes.c_int64), ("map_host_us", ctypes.c_double), ("unmap_host_us", ctypes.c_double),
+                ("tokens_appended", ctypes.c_int64), ("attention_calls", ctypes.c_int64), ("work_items", ctypes.c_int64),
+                ("partial_items", ctypes.c_int64), ("attn_launches", ctypes.c_int64), ("attn_kernel_ms", ctypes.c_double),
+                ("combine_kernel_ms", ctypes.c_double), ("append_kernel_ms", ctypes.c_double),
+                ("combine_launches", ctypes.c_int64), ("append_launches", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
+                ("sm_count", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class SlotInfo(ctypes.Structure):
+    _fields_ = [("base", ctypes.c_uint64), ("va_bytes", ctypes.c_int64), ("kv_len", ctypes.c_int64),
+                ("mapped_tokens", ctypes.c_int64), ("pages_in_range", ctypes.c_int32), ("pages_owned", ctypes.c_int32),
+                ("live", ctypes.c_int32), ("row_bytes", ctypes.c_int32)]
+
+
+class WorkItem(ctypes.Structure):
+    _fields_ = [("req", ctypes.c_int32), ("kv_head", ctypes.c_int32), ("tile_begin", ctypes.c_int32),
+                ("tile_end", ctypes.c_int32), ("q_tok0", ctypes.c_int16), ("n_q_tok", ctypes.c_int16),
+                ("g0", ctypes.c_int16), ("n_g", ctypes.c_int16), ("partial_idx", ctypes.c_int32), ("unit", ctypes.c_int32)]
+
+
+_vp, _i32p, _i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+_ctxp = ctypes.c_void_p
+
+EXPORTS = {
+    "xllm_init": (ctypes.c_int32, [ctypes.POINTER(Config), ctypes.POINTER(_ctxp)]),
+    "xllm_shutdown": (ctypes.c_int32, [_ctxp]),
+    "xllm_last_error": (ctypes.c_char_p, [_ctxp]),
+    "xllm_sync_check": (ctypes.c_int32, [_ctxp, _vp]),
+    "xllm_kv_reserve": (ctypes.c_int32, [_ctxp, ctypes.c_int64, ctypes.c_int64, _i32p]),
+    "xllm_kv_map_pages": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
+    "xllm_kv_map_pages_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i64p]),
+    "xllm_kv_set_len_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i64p]),
+    "xllm_kv_release": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int32]),
+    "xllm_kv_set_len": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
+    "xllm_kv_slot_info": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.POINTER(SlotInfo)]),
+    "xllm_kv_page_of": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, _i32p, _i32p, _i64p]),
+    "xllm_debug_read_slot": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
+    "xllm_debug_read_page": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
+    "xllm_kv_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i32p, _vp, _vp, _vp]),
+    "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
+    "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i32p, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                              ctypes.POINTER(WorkItem), ctypes.c_int32, _i32p, _i32p, _i32p, _i32p]),
+    "xllm_get_stats": (ctypes.c_int32, [_ctxp, ctypes.POINTER(Stats)]),
+    "xllm_set_profiling": (ctypes.c_int32, [_ctxp, ctypes.c_int32]),
+}
+for _name, (_res, _args) in EXPORTS.items():
+    _fn = getattr(_lib, _name)  # AttributeError here = the library does not export a declared symbol
+    _fn.restype, _fn.argtypes = _res, _args
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor / numpy array / raw int; None -> NULL."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def plan_partition(kv_lens: Sequence[int], q_lens: Optional[Sequence[int]], n_q_heads: int, n_kv_heads: int, n_ctas: int):
+    """Host-only: returns (items: list[WorkItem], cta_begin: np.ndarray, n_units, n_partials)."""
+    kv = np.ascontiguousarray(kv_lens, dtype=np.int64)
+    n = len(kv)
+    ql = _i32(q_lens) if q_lens is not None else None
+    cap = n * n_kv_heads * 16 + n_ctas + 8
+    items = (WorkItem * cap)()
+    cta = np.zeros(n_ctas + 1, np.int32)
+    n_items, n_units, n_parts = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    st = _lib.xllm_plan_partition(n, kv.ctypes.data_as(_i64p), ql.ctypes.data_as(_i32p) if ql is not None else None,
+                                  n_q_heads, n_kv_heads, n_ctas, items, cap, cta.ctypes.data_as(_i32p),
+                                  ctypes.byref(n_items), ctypes.byref(n_units), ctypes.byref(n_parts))
+    if st != OK:
+        raise XllmError(st, "xllm_plan_partition rejected the sizes")
+    return [items[i] for i in range(n_items.value)], cta, n_units.value, n_parts.value
+
+
+class Context:
+    """Owner of one ``xllm_ctx``.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, max_slots: int, max_seq_len: int,
+                 phys_budget_bytes: int, max_q_len: int = 4, device: int = 0, page_bytes: int = 0, flags: int = 0,
+                 fault_inject: int = 0):
+        self.cfg = Config(device, n_q_heads, n_kv_heads, head_dim, max_slots, max_q_len, max_seq_len, phys_budget_bytes,
+                          page_bytes, flags, fault_inject)
+        self._ctx = _ctxp()
+        st = _lib.xllm_init(ctypes.byref(self.cfg), ctypes.byref(self._ctx))
+        if st != OK:
+            self._ctx = None
+            raise XllmError(st, _lib.xllm_last_error(None).decode())
+
+    # -- plumbing --
+    def _check(self, st: int):
+        if st != OK:
+            raise XllmError(st, _lib.xllm_last_error(self._ctx).decode())
+
+    def shutdown(self):
+        if self._ctx:
+            _lib.xllm_shutdown(self._ctx)
+            self._ctx = None
+
+    close = shutdown
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.shutdown()
+
+    def __del__(self):
+        try:
+            self.shutdown()
+        except Exception:
+            pass
+
+    # -- xTensor --
+    def kv_reserve(self, max_seq_len: Optional[int] = None, expected_tokens: int = 0) -> int:
+        slot = ctypes.c_int32(-1)
+        self._check(_lib.xllm_kv_reserve(self._ctx, self.cfg.max_seq_len if max_seq_len is None else max_seq_len,
+                                         expected_tokens, ctypes.byref(slot)))
+        return slot.value
+
+    def kv_map_pages(self, slot: int, min_tokens: int):
+        self._check(_lib.xllm_kv_map_pages(self._ctx, slot, min_tokens))
+
+    def kv_map_pages_many(self, slots, min_tokens):
+        s, t = _i32(slots), np.ascontiguousarray(min_tokens, dtype=np.int64)
+        self._check(_lib.xllm_kv_map_pages_many(self._ctx, len(s), s.ctypes.data_as(_i32p), t.ctypes.data_as(_i64p)))
+
+    def kv_set_len_many(self, slots, kv_lens):
+        s, t = _i32(slots), np.ascontiguousarray(kv_lens, dtype=np.int64)
+        self._check(_lib.xllm_kv_set_len_many(self._ctx, len(s), s.ctypes.data_as(_i32p), t.ctypes.data_as(_i64p)))
+
+    def kv_release(self, slot: int, mode: int = 0):
+        self._check(_lib.xllm_kv_release(self._ctx, slot, mode))
+
+    def kv_set_len(self, slot: int, kv_len: int):
+        self._check(_lib.xllm_kv_set_len(self._ctx, slot, kv_len))
+
+    def kv_slot_info(self, slot: int) -> SlotInfo:
+        info = SlotInfo()
+        self._check(_lib.xllm_kv_slot_info(self._ctx, slot, ctypes.byref(info)))
+        return info
+
+    def kv_page_of(self, slot: int, byte_offset: int):
+        pos, pid, off = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int64()
+        self._check(_lib.xllm_kv_page_of(self._ctx, slot, byte_offset, ctypes.byref(pos), ctypes.byref(pid), ctypes.byref(off)))
+        return pos.value, pid.value, off.value
+
+    def debug_read_slot(self, slot: int, byte_offset: int, nbytes: int) -> np.ndarray:
+        buf = np.empty(nbytes, np.uint8)
+        self._check(_lib.xllm_debug_read_slot(self._ctx, slot, byte_offset, nbytes, buf.ctypes.data))
+        return buf
+
+    def debug_read_page(self, page_id: int, byte_offset: int, nbytes: int) -> np.ndarray:
+        buf = np.empty(nbytes, np.uint8)
+        self._check(_lib.xllm_debug_read_page(self._ctx, page_id, byte_offset, nbytes, buf.ctypes.data))
+        return buf
+
+    # -- KV writes --
+    def kv_append(self, slots, n_new, k_new, v_new, stream=None):
+        s, n = _i32(slots), _i32(n_new)
+        self._check(_lib.xllm_kv_append(self._ctx, len(s), s.ctypes.data_as(_i32p), n.ctypes.data_as(_i32p), _ptr(k_new),
+                                        _ptr(v_new), _stream(stream)))
+
+    def kv_gather(self, slot: int, first_token: int, n_tokens: int, k_out, v_out, stream=None):
+        self._check(_lib.xllm_kv_gather(self._ctx, slot, first_token, n_tokens, _ptr(k_out), _ptr(v_out), _stream(stream)))
+
+    # -- attention --
+    def decode_attention(self, slots, q, out, lse_out=None, scale: float = 1.0, stream=None):
+        s = _i32(slots)
+        self._check(_lib.xllm_decode_attention(self._ctx, len(s), s.ctypes.data_as(_i32p), _ptr(q), _ptr(out), _ptr(lse_out),
+                                               scale, _stream(stream)))
+
+    def verify_attention(self, slots, q_lens, q, out, lse_out=None, scale: float = 1.0, stream=None):
+        s, ql = _i32(slots), _i32(q_lens)
+        self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data_as(_i32p), ql.ctypes.data_as(_i32p), _ptr(q),
+                                               _ptr(out), _ptr(lse_out), scale, _stream(stream)))
+
+    def sync_check(self, stream=None):
+        self._check(_lib.xllm_sync_check(self._ctx, _stream(stream)))
+
+    # -- statistics --
+    def get_stats(self) -> Stats:
+        st = Stats()
+        self._check(_lib.xllm_get_stats(self._ctx, ctypes.byref(st)))
+        return st
+
+    def set_profiling(self, on: bool):
+        self._check(_lib.xllm_set_profiling(self._ctx, 1 if on else 0))

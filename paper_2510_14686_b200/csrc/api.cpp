@@ -1,0 +1,661 @@
+// C ABI of libxllm_attn.so: argument checks, host bookkeeping, work-list staging and kernel launches.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "xllm_attn.h"
+#include "xllm_internal.h"
+#include "xtensor.h"
+
+using namespace xllm;
+
+namespace {
+
+constexpr int kRing = 16;  // staging buffers / completion events kept in flight
+
+struct TimedLaunch {
+    cudaEvent_t start, stop;
+    int kind;  // 0 attention, 1 combine, 2 append
+};
+
+thread_local std::string g_init_error;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct xllm_ctx {
+    xllm_config cfg{};
+    std::unique_ptr<XTensor> xt;
+    bool host_only = false;
+    int sm_count = 0;
+    std::string err;
+    PlanTuning tune;
+
+    // staging ring: pinned host buffers, one device copy target each, one completion event each
+    size_t stage_bytes = 0;
+    char *h_stage[kRing] = {};
+    char *d_stage[kRing] = {};
+    cudaEvent_t done[kRing] = {};
+    bool done_recorded[kRing] = {};
+    uint64_t seq = 0;        // launches so far (1-based sequence numbers)
+    cudaStream_t last_stream = nullptr;
+
+    float *d_part_o = nullptr, *d_part_lse = nullptr;
+    int32_t max_partials = 0, max_items = 0;
+    int32_t *h_error = nullptr, *d_error = nullptr;  // mapped pinned word written by kernels whose waits expired
+
+    // scratch for debug_read_page
+    uint64_t scratch_va = 0;
+
+    bool profiling = false;
+    std::vector<TimedLaunch> timed;
+    std::vector<cudaEvent_t> event_pool;
+    xllm_stats st{};
+
+    std::vector<xllm_work_item> items;
+    std::vector<int32_t> cta_begin;
+    std::vector<int64_t> kv_lens;
+    std::vector<uint8_t> seen;
+};
+
+namespace {
+
+xllm_status fail(xllm_ctx *ctx, xllm_status code, const std::string &msg) {
+    if (ctx) ctx->err = msg;
+    return code;
+}
+
+xllm_status cuda_fail(xllm_ctx *ctx, const char *what, int e) {
+    return fail(ctx, XLLM_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString((cudaError_t)e));
+}
+
+// Reports a device-side wait that gave up, if any kernel flagged one since the last check.
+xllm_status check_device_flag(xllm_ctx *ctx) {
+    if (ctx->h_error && *reinterpret_cast<volatile int32_t *>(ctx->h_error) != 0) {
+        const int code = *ctx->h_error;
+        *ctx->h_error = 0;
+        return fail(ctx, XLLM_ERR_CUDA, "attention kernel: a bounded device-side wait expired (code " + std::to_string(code) +
+                                            "); the results of that launch are invalid");
+    }
+    return XLLM_OK;
+}
+
+cudaEvent_t get_event(xllm_ctx *ctx) {
+    if (!ctx->event_pool.empty()) {
+        cudaEvent_t e = ctx->event_pool.back();
+        ctx->event_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+void time_begin(xllm_ctx *ctx, int kind, cudaStream_t st) {
+    if (!ctx->profiling) return;
+    TimedLaunch t{get_event(ctx), get_event(ctx), kind};
+    cudaEventRecord(t.start, st);
+    ctx->timed.push_back(t);
+}
+void time_end(xllm_ctx *ctx, cudaStream_t st) {
+    if (!ctx->profiling) return;
+    cudaEventRecord(ctx->timed.back().stop, st);
+}
+
+void resolve_timings(xllm_ctx *ctx) {
+    for (TimedLaunch &t : ctx->timed) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(t.stop) == cudaSuccess && cudaEventElapsedTime(&ms, t.start, t.stop) == cudaSuccess) {
+            if (t.kind == 0) { ctx->st.attn_kernel_ms += ms; ++ctx->st.attn_launches; }
+            else if (t.kind == 1) { ctx->st.combine_kernel_ms += ms; ++ctx->st.combine_launches; }
+            else { ctx->st.append_kernel_ms += ms; ++ctx->st.append_launches; }
+        }
+        ctx->event_pool.push_back(t.start);
+        ctx->event_pool.push_back(t.stop);
+    }
+    ctx->timed.clear();
+}
+
+// Next staging buffer; waits (normally not at all) until the copy that last used it has completed.
+int acquire_stage(xllm_ctx *ctx, int *idx) {
+    const int i = (int)(ctx->seq % kRing);
+    if (ctx->done_recorded[i]) {
+        const cudaError_t e = cudaEventSynchronize(ctx->done[i]);
+        if (e != cudaSuccess) return (int)e;
+    }
+    *idx = i;
+    return 0;
+}
+
+void finish_launch(xllm_ctx *ctx, int idx, cudaStream_t st) {
+    cudaEventRecord(ctx->done[idx], st);
+    ctx->done_recorded[idx] = true;
+    ++ctx->seq;
+    ctx->last_stream = st;
+}
+
+// 0 when nothing in flight can still touch the slot.
+int wait_slot_idle(xllm_ctx *ctx, const SlotRecord &s) {
+    if (ctx->host_only || s.last_use == 0) return 0;
+    const uint64_t use = s.last_use;  // 1-based sequence number of the launch
+    // Launch n + kRing re-used launch n's staging buffer and waited for n's completion event first, so anything
+    // at least kRing launches old is known to have finished.
+    if (use + kRing <= ctx->seq) return 0;
+    const int i = (int)((use - 1) % kRing);
+    if (!ctx->done_recorded[i]) return 0;
+    if (ctx->cfg.flags & XLLM_FLAG_NONBLOCKING_UNMAP)
+        return cudaEventQuery(ctx->done[i]) == cudaSuccess ? 0 : XLLM_ERR_BUSY;
+    return cudaEventSynchronize(ctx->done[i]) == cudaSuccess ? 0 : XLLM_ERR_CUDA;
+}
+
+xllm_status check_slot_list(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const char *who) {
+    if (n_req < 1 || !slots) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": n_req must be >= 1 and slots non-null");
+    if (n_req > ctx->cfg.max_slots) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": more requests than slots");
+    ctx->seen.assign((size_t)ctx->cfg.max_slots, 0);
+    for (int32_t i = 0; i < n_req; ++i) {
+        const int32_t s = slots[i];
+        if (!ctx->xt->valid_slot(s) || !ctx->xt->slot(s).live)
+            return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(s) + " is not live");
+        if (ctx->seen[(size_t)s]) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(s) + " listed twice");
+        ctx->seen[(size_t)s] = 1;
+    }
+    return XLLM_OK;
+}
+
+xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
+                           void *out, float *lse_out, float scale, void *cuda_stream, const char *who) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context is host-only, no GPU work possible");
+    xllm_status st = check_device_flag(ctx);
+    if (st != XLLM_OK) return st;
+    st = check_slot_list(ctx, n_req, slots, who);
+    if (st != XLLM_OK) return st;
+    if (!q || !out) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q and out must be non-null device pointers");
+    if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q and out must be 16-byte aligned");
+    if (!(scale > 0.f) || !std::isfinite(scale)) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": scale must be finite and > 0");
+
+    ctx->kv_lens.resize((size_t)n_req);
+    int64_t q_rows = 0;
+    for (int32_t i = 0; i < n_req; ++i) {
+        const int32_t ql = q_lens ? q_lens[i] : 1;
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        if (ql < 1 || ql > ctx->cfg.max_q_len)
+            return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q_len of request " + std::to_string(i) + " outside [1, max_q_len]");
+        if (s.kv_len < ql)
+            return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(slots[i]) + " holds " +
+                                                   std::to_string(s.kv_len) + " tokens, fewer than q_len " + std::to_string(ql));
+        ctx->kv_lens[(size_t)i] = s.kv_len;
+        q_rows += ql;
+    }
+    int32_t n_units = 0, n_partials = 0;
+    if (plan_partition(n_req, ctx->kv_lens.data(), q_lens, ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, ctx->sm_count, ctx->tune,
+                       ctx->items, ctx->cta_begin, &n_units, &n_partials) != 0)
+        return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
+    const int32_t n_items = (int32_t)ctx->items.size();
+    if (n_items > ctx->max_items || n_partials > ctx->max_partials)
+        return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": work list exceeds the workspace sized at init");
+
+    // split units -> combine descriptors (a unit's partials are consecutive)
+    std::vector<CombineDesc> combine;
+    const int32_t G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
+    std::vector<int32_t> q_row0((size_t)n_req);
+    {
+        int32_t acc = 0;
+        for (int32_t i = 0; i < n_req; ++i) {
+            q_row0[(size_t)i] = acc;
+            acc += q_lens ? q_lens[i] : 1;
+        }
+    }
+    int32_t last_unit = -1;
+    for (const xllm_work_item &it : ctx->items) {
+        if (it.partial_idx < 0) continue;
+        if (it.unit == last_unit) {
+            ++combine.back().n_parts;
+        } else {
+            combine.push_back({it.partial_idx, 1, q_row0[(size_t)it.req] + it.q_tok0, it.kv_head * G + it.g0, it.n_q_tok, it.n_g});
+            last_unit = it.unit;
+        }
+    }
+
+    int idx;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    // layout of the staged blob
+    const size_t off_items = 0;
+    const size_t off_cta = align_up(off_items + sizeof(xllm_work_item) * (size_t)n_items, 16);
+    const size_t off_reqs = align_up(off_cta + sizeof(int32_t) * (size_t)(ctx->sm_count + 1), 16);
+    const size_t off_comb = align_up(off_reqs + sizeof(ReqDesc) * (size_t)n_req, 16);
+    const size_t total = align_up(off_comb + sizeof(CombineDesc) * combine.size(), 16);
+    if (total > ctx->stage_bytes) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
+    char *h = ctx->h_stage[idx];
+    std::memcpy(h + off_items, ctx->items.data(), sizeof(xllm_work_item) * (size_t)n_items);
+    std::memcpy(h + off_cta, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    ReqDesc *rd = reinterpret_cast<ReqDesc *>(h + off_reqs);
+    for (int32_t i = 0; i < n_req; ++i) {
+        SlotRecord &s = ctx->xt->slot(slots[i]);
+        rd[i].base = s.base;
+        rd[i].kv_len = (int32_t)s.kv_len;
+        rd[i].q_len = q_lens ? q_lens[i] : 1;
+        rd[i].q_row0 = q_row0[(size_t)i];
+        rd[i].pad = 0;
+    }
+    if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    char *d = ctx->d_stage[idx];
+    e = (int)cudaMemcpyAsync(d, h, total, cudaMemcpyHostToDevice, stream);
+    if (e) return cuda_fail(ctx, "staging the work list", e);
+
+    AttnLaunch al{};
+    al.items = reinterpret_cast<const xllm_work_item *>(d + off_items);
+    al.cta_begin = reinterpret_cast<const int32_t *>(d + off_cta);
+    al.reqs = reinterpret_cast<const ReqDesc *>(d + off_reqs);
+    al.q = q;
+    al.out = out;
+    al.lse_out = lse_out;
+    al.part_o = ctx->d_part_o;
+    al.part_lse = ctx->d_part_lse;
+    al.error_flag = ctx->d_error;
+    al.n_q_heads = ctx->cfg.n_q_heads;
+    al.n_kv_heads = ctx->cfg.n_kv_heads;
+    al.head_dim = ctx->cfg.head_dim;
+    al.scale_log2 = scale * 1.4426950408889634f;
+    al.n_ctas = ctx->sm_count;
+    time_begin(ctx, 0, stream);
+    e = launch_attention(al, stream);
+    time_end(ctx, stream);
+    if (e) return cuda_fail(ctx, "launching the attention kernel", e);
+    ++ctx->st.kernel_launches;
+    if (!combine.empty()) {
+        CombineLaunch cl{};
+        cl.descs = reinterpret_cast<const CombineDesc *>(d + off_comb);
+        cl.n_units = (int32_t)combine.size();
+        cl.part_o = ctx->d_part_o;
+        cl.part_lse = ctx->d_part_lse;
+        cl.out = out;
+        cl.lse_out = lse_out;
+        cl.n_q_heads = ctx->cfg.n_q_heads;
+        cl.head_dim = ctx->cfg.head_dim;
+        time_begin(ctx, 1, stream);
+        e = launch_combine(cl, stream);
+        time_end(ctx, stream);
+        if (e) return cuda_fail(ctx, "launching the combine kernel", e);
+        ++ctx->st.kernel_launches;
+    }
+    finish_launch(ctx, idx, stream);
+    for (int32_t i = 0; i < n_req; ++i) ctx->xt->slot(slots[i]).last_use = ctx->seq;
+    ++ctx->st.attention_calls;
+    ctx->st.work_items += n_items;
+    ctx->st.partial_items += n_partials;
+    return XLLM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
+    if (!cfg || !out) {
+        g_init_error = "xllm_init: null argument";
+        return XLLM_ERR_INVALID;
+    }
+    *out = nullptr;
+    auto bad = [&](xllm_status code, const std::string &m) {
+        g_init_error = "xllm_init: " + m;
+        return code;
+    };
+    if (cfg->n_kv_heads < 1 || cfg->n_q_heads < cfg->n_kv_heads || cfg->n_q_heads % cfg->n_kv_heads)
+        return bad(XLLM_ERR_INVALID, "n_q_heads must be a positive multiple of n_kv_heads");
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return bad(XLLM_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    if (cfg->max_slots < 1 || cfg->max_seq_len < 1 || cfg->max_seq_len > (int64_t)INT32_MAX - XLLM_TILE_TOKENS)
+        return bad(XLLM_ERR_INVALID, "max_slots and max_seq_len must be positive (max_seq_len < 2^31)");
+    if (cfg->max_q_len < 1 || cfg->max_q_len > XLLM_MAX_Q_LEN) return bad(XLLM_ERR_INVALID, "max_q_len must be in [1, XLLM_MAX_Q_LEN]");
+    if (cfg->phys_budget_bytes < 1 || cfg->page_bytes < 0) return bad(XLLM_ERR_INVALID, "phys_budget_bytes must be positive, page_bytes >= 0");
+
+    std::unique_ptr<xllm_ctx> ctx(new xllm_ctx());
+    ctx->cfg = *cfg;
+    ctx->host_only = (cfg->flags & XLLM_FLAG_HOST_ONLY) != 0;
+    const int64_t row_bytes = 2ll * cfg->n_kv_heads * cfg->head_dim * 2;
+    std::unique_ptr<VmmDriver> drv;
+    if (ctx->host_only) {
+        drv = make_fake_driver(cfg->fault_inject);
+        ctx->sm_count = 148;
+    } else {
+        int n_dev = 0;
+        cudaError_t e = cudaGetDeviceCount(&n_dev);
+        if (e != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev)
+            return bad(XLLM_ERR_CUDA, std::string("no such CUDA device (") + cudaGetErrorString(e) +
+                                          "); this library has no CPU fallback");
+        if ((e = cudaSetDevice(cfg->device)) != cudaSuccess || (e = cudaFree(nullptr)) != cudaSuccess)
+            return bad(XLLM_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e));
+        cudaDeviceProp prop;
+        cudaGetDeviceProperties(&prop, cfg->device);
+        if (prop.major != 10) return bad(XLLM_ERR_UNSUPPORTED, "kernels are built for sm_100a only; device is sm_" +
+                                                                  std::to_string(prop.major) + std::to_string(prop.minor));
+        ctx->sm_count = prop.multiProcessorCount;
+        std::string derr;
+        drv = make_cuda_driver(&derr);
+        if (!drv) return bad(XLLM_ERR_CUDA, derr);
+    }
+    ctx->xt.reset(new XTensor(std::move(drv), cfg->device, cfg->max_slots, cfg->max_seq_len, row_bytes));
+    std::string perr;
+    xllm_status st = ctx->xt->init_pool(cfg->phys_budget_bytes, cfg->page_bytes, (cfg->flags & XLLM_FLAG_LAZY_PAGES) != 0, &perr);
+    if (st != XLLM_OK) return bad(st, perr);
+    if (ctx->xt->page_bytes() % ((int64_t)XLLM_TILE_TOKENS * row_bytes) != 0 &&
+        ((int64_t)XLLM_TILE_TOKENS * row_bytes) % ctx->xt->page_bytes() != 0)
+        return bad(XLLM_ERR_UNSUPPORTED, "page size and tile block size must divide one another");
+    xllm_ctx *raw = ctx.get();
+    ctx->xt->wait_idle = [raw](const SlotRecord &s) { return wait_slot_idle(raw, s); };
+
+    // workspace sized for the largest call: every slot once, every row group, plus one item per CTA cut
+    const int32_t G = cfg->n_q_heads / cfg->n_kv_heads;
+    const int32_t groups = (G <= kMaxRows) ? (cfg->max_q_len + std::max(1, kMaxRows / G) - 1) / std::max(1, kMaxRows / G)
+                                           : cfg->max_q_len * ((G + kMaxRows - 1) / kMaxRows);
+    ctx->max_items = cfg->max_slots * cfg->n_kv_heads * groups + ctx->sm_count + 1;
+    ctx->max_partials = 2 * ctx->sm_count + 2;
+    ctx->stage_bytes = align_up(sizeof(xllm_work_item) * (size_t)ctx->max_items, 16) +
+                       align_up(sizeof(int32_t) * (size_t)(ctx->sm_count + 1), 16) +
+                       align_up(std::max(sizeof(ReqDesc), sizeof(AppendDesc)) * (size_t)cfg->max_slots, 16) +
+                       align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16) + 64;
+    if (!ctx->host_only) {
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < kRing && e == cudaSuccess; ++i) {
+            e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_stage[i]), ctx->stage_bytes, cudaHostAllocDefault);
+            if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_stage[i]), ctx->stage_bytes);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->done[i], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * kMaxRows * cfg->head_dim);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * kMaxRows);
+        if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_error), sizeof(int32_t), cudaHostAllocMapped);
+        if (e == cudaSuccess) {
+            *ctx->h_error = 0;
+            e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&ctx->d_error), ctx->h_error, 0);
+        }
+        if (e == cudaSuccess) e = (cudaError_t)configure_kernels(cfg->head_dim);
+        if (e != cudaSuccess) {
+            const std::string m = std::string("allocating the workspace: ") + cudaGetErrorString(e);
+            xllm_shutdown(ctx.release());
+            return bad(XLLM_ERR_CUDA, m);
+        }
+    }
+    ctx->st.sm_count = ctx->sm_count;
+    *out = ctx.release();
+    return XLLM_OK;
+}
+
+xllm_status xllm_shutdown(xllm_ctx *ctx) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (!ctx->host_only) {
+        cudaSetDevice(ctx->cfg.device);
+        cudaDeviceSynchronize();
+    }
+    if (ctx->scratch_va) ctx->xt->driver().free_va(ctx->scratch_va, (size_t)ctx->xt->page_bytes());
+    if (ctx->xt) ctx->xt->teardown();
+    if (!ctx->host_only) {
+        for (int i = 0; i < kRing; ++i) {
+            if (ctx->h_stage[i]) cudaFreeHost(ctx->h_stage[i]);
+            if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
+            if (ctx->done[i]) cudaEventDestroy(ctx->done[i]);
+        }
+        if (ctx->d_part_o) cudaFree(ctx->d_part_o);
+        if (ctx->d_part_lse) cudaFree(ctx->d_part_lse);
+        if (ctx->h_error) cudaFreeHost(ctx->h_error);
+        for (TimedLaunch &t : ctx->timed) {
+            cudaEventDestroy(t.start);
+            cudaEventDestroy(t.stop);
+        }
+        for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
+    }
+    delete ctx;
+    return XLLM_OK;
+}
+
+const char *xllm_last_error(const xllm_ctx *ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+xllm_status xllm_sync_check(xllm_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return XLLM_OK;
+    const cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, "cudaStreamSynchronize", (int)e);
+    return check_device_flag(ctx);
+}
+
+xllm_status xllm_kv_reserve(xllm_ctx *ctx, int64_t max_seq_len, int64_t expected_tokens, int32_t *slot_out) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    return ctx->xt->reserve(max_seq_len, expected_tokens, slot_out, &ctx->err);
+}
+
+xllm_status xllm_kv_map_pages(xllm_ctx *ctx, int32_t slot, int64_t min_tokens) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    return ctx->xt->map_pages(slot, min_tokens, &ctx->err);
+}
+
+xllm_status xllm_kv_map_pages_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (n_req < 0 || !slots || !min_tokens) return fail(ctx, XLLM_ERR_INVALID, "map_pages_many: null argument");
+    for (int32_t i = 0; i < n_req; ++i) {
+        const xllm_status st = ctx->xt->map_pages(slots[i], min_tokens[i], &ctx->err);
+        if (st != XLLM_OK) return st;
+    }
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_release(xllm_ctx *ctx, int32_t slot, int32_t mode) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    return ctx->xt->release(slot, mode, &ctx->err);
+}
+
+xllm_status xllm_kv_set_len(xllm_ctx *ctx, int32_t slot, int64_t kv_len) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "set_len: slot is not live");
+    if (kv_len < 0 || kv_len > ctx->xt->mapped_tokens(slot) || kv_len > ctx->cfg.max_seq_len)
+        return fail(ctx, XLLM_ERR_INVALID, "set_len: kv_len must lie in [0, mapped tokens]");
+    ctx->xt->slot(slot).kv_len = kv_len;
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_set_len_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *kv_lens) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (n_req < 0 || !slots || !kv_lens) return fail(ctx, XLLM_ERR_INVALID, "set_len_many: null argument");
+    for (int32_t i = 0; i < n_req; ++i) {
+        if (!ctx->xt->valid_slot(slots[i]) || !ctx->xt->slot(slots[i]).live)
+            return fail(ctx, XLLM_ERR_INVALID, "set_len_many: slot " + std::to_string(slots[i]) + " is not live");
+        if (kv_lens[i] < 0 || kv_lens[i] > ctx->xt->mapped_tokens(slots[i]) || kv_lens[i] > ctx->cfg.max_seq_len)
+            return fail(ctx, XLLM_ERR_INVALID, "set_len_many: kv_len must lie in [0, mapped tokens]");
+    }
+    for (int32_t i = 0; i < n_req; ++i) ctx->xt->slot(slots[i]).kv_len = kv_lens[i];
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_slot_info(const xllm_ctx *ctx, int32_t slot, xllm_slot_info *info) {
+    if (!ctx || !info || !ctx->xt->valid_slot(slot)) return XLLM_ERR_INVALID;
+    const SlotRecord &s = ctx->xt->slot(slot);
+    info->base = s.base;
+    info->va_bytes = ctx->xt->va_bytes();
+    info->kv_len = s.kv_len;
+    info->mapped_tokens = ctx->xt->mapped_tokens(slot);
+    info->pages_in_range = (int32_t)s.pages.size();
+    info->pages_owned = s.n_owned;
+    info->live = s.live ? 1 : 0;
+    info->row_bytes = (int32_t)ctx->xt->row_bytes();
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_page_of(const xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int32_t *page_pos, int32_t *page_id,
+                            int64_t *in_page_offset) {
+    if (!ctx || !ctx->xt->valid_slot(slot) || byte_offset < 0 || byte_offset >= ctx->xt->va_bytes()) return XLLM_ERR_INVALID;
+    const SlotRecord &s = ctx->xt->slot(slot);
+    const int64_t pos = byte_offset / ctx->xt->page_bytes();
+    if (pos >= (int64_t)s.pages.size()) return XLLM_ERR_NOT_MAPPED;
+    if (page_pos) *page_pos = (int32_t)pos;
+    if (page_id) *page_id = s.pages[(size_t)pos];
+    if (in_page_offset) *in_page_offset = byte_offset % ctx->xt->page_bytes();
+    return XLLM_OK;
+}
+
+xllm_status xllm_debug_read_slot(xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int64_t nbytes, void *host_dst) {
+    if (!ctx || !host_dst) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_slot: host-only context");
+    if (!ctx->xt->valid_slot(slot) || byte_offset < 0 || nbytes < 0) return fail(ctx, XLLM_ERR_INVALID, "debug_read_slot: bad arguments");
+    const SlotRecord &s = ctx->xt->slot(slot);
+    if (byte_offset + nbytes > (int64_t)s.pages.size() * ctx->xt->page_bytes())
+        return fail(ctx, XLLM_ERR_NOT_MAPPED, "debug_read_slot: range is not fully mapped");
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(host_dst, reinterpret_cast<const void *>(s.base + (uint64_t)byte_offset), (size_t)nbytes, cudaMemcpyDeviceToHost);
+    return e == cudaSuccess ? XLLM_OK : cuda_fail(ctx, "debug_read_slot", (int)e);
+}
+
+xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_offset, int64_t nbytes, void *host_dst) {
+    if (!ctx || !host_dst) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_page: host-only context");
+    const int64_t pb = ctx->xt->page_bytes();
+    if (page_id < 0 || page_id >= (int32_t)ctx->xt->pages().size() || byte_offset < 0 || nbytes < 0 || byte_offset + nbytes > pb)
+        return fail(ctx, XLLM_ERR_INVALID, "debug_read_page: bad arguments");
+    const PageRecord &pr = ctx->xt->pages()[(size_t)page_id];
+    if (!pr.created) return fail(ctx, XLLM_ERR_NOT_MAPPED, "debug_read_page: the page has no physical memory yet");
+    VmmDriver &drv = ctx->xt->driver();
+    if (!ctx->scratch_va && (drv.reserve(&ctx->scratch_va, (size_t)pb, (size_t)pb) != 0 || !ctx->scratch_va)) {
+        ctx->scratch_va = 0;
+        return fail(ctx, XLLM_ERR_OOM_VA, "debug_read_page: could not reserve a scratch range");
+    }
+    cudaDeviceSynchronize();
+    if (drv.map(ctx->scratch_va, (size_t)pb, pr.handle) != 0) return fail(ctx, XLLM_ERR_CUDA, "debug_read_page: cuMemMap failed");
+    xllm_status st = XLLM_OK;
+    if (drv.set_access(ctx->scratch_va, (size_t)pb, ctx->cfg.device) != 0) st = fail(ctx, XLLM_ERR_CUDA, "debug_read_page: cuMemSetAccess failed");
+    if (st == XLLM_OK) {
+        const cudaError_t e = cudaMemcpy(host_dst, reinterpret_cast<const void *>(ctx->scratch_va + (uint64_t)byte_offset), (size_t)nbytes, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) st = cuda_fail(ctx, "debug_read_page", (int)e);
+    }
+    drv.unmap(ctx->scratch_va, (size_t)pb);
+    return st;
+}
+
+xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new, const void *k_new,
+                           const void *v_new, void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "append: context is host-only, no GPU work possible");
+    xllm_status st = check_device_flag(ctx);
+    if (st != XLLM_OK) return st;
+    st = check_slot_list(ctx, n_req, slots, "append");
+    if (st != XLLM_OK) return st;
+    if (!n_new || !k_new || !v_new) return fail(ctx, XLLM_ERR_INVALID, "append: null argument");
+    if ((reinterpret_cast<uintptr_t>(k_new) & 15) || (reinterpret_cast<uintptr_t>(v_new) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, "append: k_new and v_new must be 16-byte aligned");
+    int64_t rows = 0;
+    for (int32_t i = 0; i < n_req; ++i) {
+        if (n_new[i] < 0) return fail(ctx, XLLM_ERR_INVALID, "append: negative n_new");
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        if (s.kv_len + n_new[i] > ctx->cfg.max_seq_len)
+            return fail(ctx, XLLM_ERR_INVALID, "append: slot " + std::to_string(slots[i]) + " would exceed max_seq_len");
+        if (s.kv_len + n_new[i] > ctx->xt->mapped_tokens(slots[i]))
+            return fail(ctx, XLLM_ERR_NOT_MAPPED, "append: slot " + std::to_string(slots[i]) + " has pages for " +
+                                                      std::to_string(ctx->xt->mapped_tokens(slots[i])) + " tokens, needs " +
+                                                      std::to_string(s.kv_len + n_new[i]) + "; call xllm_kv_map_pages first");
+        rows += n_new[i];
+    }
+    if (rows > INT32_MAX) return fail(ctx, XLLM_ERR_INVALID, "append: too many rows");
+    if (rows == 0) return XLLM_OK;
+    int idx;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    AppendDesc *ad = reinterpret_cast<AppendDesc *>(ctx->h_stage[idx]);
+    int32_t row0 = 0, n_desc = 0;
+    for (int32_t i = 0; i < n_req; ++i) {
+        if (n_new[i] == 0) continue;
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        ad[n_desc++] = {s.base, (int32_t)s.kv_len, row0, n_new[i], 0};
+        row0 += n_new[i];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    e = (int)cudaMemcpyAsync(ctx->d_stage[idx], ad, sizeof(AppendDesc) * (size_t)n_desc, cudaMemcpyHostToDevice, stream);
+    if (e) return cuda_fail(ctx, "staging the append list", e);
+    time_begin(ctx, 2, stream);
+    e = launch_append(reinterpret_cast<const AppendDesc *>(ctx->d_stage[idx]), n_desc, (int32_t)rows, k_new, v_new,
+                      ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);
+    time_end(ctx, stream);
+    if (e) return cuda_fail(ctx, "launching the append kernel", e);
+    ++ctx->st.kernel_launches;
+    finish_launch(ctx, idx, stream);
+    for (int32_t i = 0; i < n_req; ++i) {
+        SlotRecord &s = ctx->xt->slot(slots[i]);
+        s.kv_len += n_new[i];
+        s.last_use = ctx->seq;
+    }
+    ctx->st.tokens_appended += rows;
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out,
+                           void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "gather: context is host-only, no GPU work possible");
+    if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "gather: slot is not live");
+    if (!k_out || !v_out || (reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, "gather: outputs must be non-null and 16-byte aligned");
+    SlotRecord &s = ctx->xt->slot(slot);
+    if (first_token < 0 || n_tokens < 0 || first_token + n_tokens > s.kv_len)
+        return fail(ctx, XLLM_ERR_INVALID, "gather: token range outside [0, kv_len)");
+    if (n_tokens == 0) return XLLM_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int idx;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    e = launch_gather(s.base, first_token, n_tokens, k_out, v_out, ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);
+    if (e) return cuda_fail(ctx, "launching the gather kernel", e);
+    ++ctx->st.kernel_launches;
+    finish_launch(ctx, idx, stream);
+    s.last_use = ctx->seq;
+    return XLLM_OK;
+}
+
+xllm_status xllm_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const void *q, void *out, float *lse_out,
+                                  float scale, void *cuda_stream) {
+    return attention_impl(ctx, n_req, slots, nullptr, q, out, lse_out, scale, cuda_stream, "decode_attention");
+}
+
+xllm_status xllm_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
+                                  void *out, float *lse_out, float scale, void *cuda_stream) {
+    if (ctx && !q_lens) return fail(ctx, XLLM_ERR_INVALID, "verify_attention: q_lens must be non-null");
+    return attention_impl(ctx, n_req, slots, q_lens, q, out, lse_out, scale, cuda_stream, "verify_attention");
+}
+
+xllm_status xllm_plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
+                                int32_t n_kv_heads, int32_t n_ctas, xllm_work_item *items, int32_t max_items, int32_t *cta_begin,
+                                int32_t *n_items_out, int32_t *n_units_out, int32_t *n_partials_out) {
+    if (!kv_lens || !items || !cta_begin || max_items < 0) return XLLM_ERR_INVALID;
+    std::vector<xllm_work_item> v;
+    std::vector<int32_t> cb;
+    PlanTuning tune;
+    if (plan_partition(n_req, kv_lens, q_lens, n_q_heads, n_kv_heads, n_ctas, tune, v, cb, n_units_out, n_partials_out) != 0)
+        return XLLM_ERR_INVALID;
+    if ((int64_t)v.size() > max_items) return XLLM_ERR_INVALID;
+    std::memcpy(items, v.data(), sizeof(xllm_work_item) * v.size());
+    std::memcpy(cta_begin, cb.data(), sizeof(int32_t) * cb.size());
+    if (n_items_out) *n_items_out = (int32_t)v.size();
+    return XLLM_OK;
+}
+
+xllm_status xllm_get_stats(const xllm_ctx *ctx_c, xllm_stats *stats) {
+    if (!ctx_c || !stats) return XLLM_ERR_INVALID;
+    xllm_ctx *ctx = const_cast<xllm_ctx *>(ctx_c);
+    if (!ctx->host_only) resolve_timings(ctx);
+    ctx->xt->fill_stats(&ctx->st);
+    *stats = ctx->st;
+    return XLLM_OK;
+}
+
+xllm_status xllm_set_profiling(xllm_ctx *ctx, int32_t on) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    ctx->profiling = on != 0 && !ctx->host_only;
+    return XLLM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+// Private declarations shared by the host files and the CUDA kernels of libxllm_attn.so.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "xllm_attn.h"
+
+namespace xllm {
+
+constexpr int32_t kMaxRows = 16;  // query rows (heads of a GQA group x query tokens) one work item carries
+
+struct PlanTuning {
+    int32_t tile_cost = 4;        // cost of one KV tile block on the partition axis
+    int32_t unit_overhead = 3;    // fixed cost of starting a unit (Q load, merge, output), same scale
+    int32_t min_piece_tiles = 4;  // pieces of a split unit are at least this many tiles
+};
+
+int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
+                   int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
+                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out);
+
+// ---- slot layout (private to the library) -----------------------------------------------------------
+// A slot's range is a sequence of tile blocks of XLLM_TILE_TOKENS tokens.  A tile block holds, for each
+// KV head in turn, a "head tile": K then V, each stored as head_dim/64 panels of [64 tokens][64 dims]
+// bf16 (128 B per token row), with the eight 16-byte chunks of a row XOR-swizzled by (token & 7).
+// A head tile is therefore one contiguous run that lands in shared memory with a few linear bulk
+// copies and can be fed to ldmatrix without bank conflicts.
+constexpr int32_t kPanelBytes = XLLM_TILE_TOKENS * 128;  // 8 KiB
+
+inline int64_t head_tile_bytes(int32_t head_dim) { return 2ll * (head_dim / 64) * kPanelBytes; }
+inline int64_t tile_block_bytes(int32_t n_kv_heads, int32_t head_dim) { return n_kv_heads * head_tile_bytes(head_dim); }
+
+// ---- device-side records ------------------------------------------------------------------------------
+struct ReqDesc {            // one per request of an attention call
+    uint64_t base;          // slot range start
+    int32_t kv_len;
+    int32_t q_len;
+    int32_t q_row0;         // first row of the request in q / out
+    int32_t pad;
+};
+
+struct CombineDesc {        // one per split unit
+    int32_t partial_begin, n_parts;
+    int32_t out_row0;       // q_row0 + q_tok0
+    int32_t head0;          // kv_head * G + g0
+    int32_t n_q_tok, n_g;
+};
+
+struct AppendDesc {         // one per request of an append / gather call
+    uint64_t base;
+    int32_t pos0;           // first token position written
+    int32_t row0;           // first source row
+    int32_t n_new;
+    int32_t pad;
+};
+
+struct AttnLaunch {
+    const xllm_work_item *items;  // device
+    const int32_t *cta_begin;     // device [n_ctas + 1]
+    const ReqDesc *reqs;          // device
+    const void *q;
+    void *out;
+    float *lse_out;               // may be null
+    float *part_o;                // [n_partials][kMaxRows][D] fp32
+    float *part_lse;              // [n_partials][kMaxRows]    (log2 domain)
+    int32_t *error_flag;          // device; set non-zero when a bounded wait expires
+    int32_t n_q_heads, n_kv_heads, head_dim;
+    float scale_log2;             // scale * log2(e)
+    int32_t n_ctas;
+};
+
+struct CombineLaunch {
+    const CombineDesc *descs;  // device
+    int32_t n_units;
+    const float *part_o;
+    const float *part_lse;
+    void *out;
+    float *lse_out;
+    int32_t n_q_heads, head_dim;
+};
+
+// kernels.cu
+int attention_smem_bytes(int32_t head_dim);
+int configure_kernels(int32_t head_dim);  // cudaFuncSetAttribute for the dynamic shared memory; returns cudaError
+int launch_attention(const AttnLaunch &p, void *stream);
+int launch_combine(const CombineLaunch &p, void *stream);
+int launch_append(const AppendDesc *descs, int32_t n_req, int32_t n_rows, const void *k_new, const void *v_new,
+                  int32_t n_kv_heads, int32_t head_dim, void *stream);
+int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,
+                  int32_t head_dim, void *stream);
+
+}  // namespace xllm

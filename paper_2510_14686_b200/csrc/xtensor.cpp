@@ -1,0 +1,481 @@
+// xTensor mapper (host): see xtensor.h.  Follows the report's "Efficient Memory Management" section:
+// fixed-size physical pages created up front, each tracked as <PageID, Status, OwnerSession>; one virtual
+// range of MaxSeqLen per request slot, reserved without backing; pages mapped on demand at the next
+// contiguous position as the sequence grows; finished requests leave their pages mapped as Reusable so a
+// later request taking the slot over needs no Map/Unmap.
+#include "xtensor.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <chrono>
+#include <cstring>
+#include <map>
+
+#include "xllm_internal.h"
+
+namespace xllm {
+
+namespace {
+
+double now_us() {
+    return std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+// ---- the real thing: CUDA VMM driver entry points, resolved through the runtime (no link-time libcuda) ----
+class CudaDriver final : public VmmDriver {
+  public:
+    bool load(std::string *err) {
+        return get("cuMemGetAllocationGranularity", &granularity_, err) && get("cuMemAddressReserve", &reserve_, err) &&
+               get("cuMemAddressFree", &free_, err) && get("cuMemCreate", &create_, err) &&
+               get("cuMemRelease", &release_, err) && get("cuMemMap", &map_, err) &&
+               get("cuMemSetAccess", &set_access_, err) && get("cuMemUnmap", &unmap_, err);
+    }
+    int granularity(int device, size_t *out) override {
+        CUmemAllocationProp prop = make_prop(device);
+        return (int)granularity_(out, &prop, CU_MEM_ALLOC_GRANULARITY_MINIMUM);
+    }
+    int reserve(uint64_t *va, size_t size, size_t align) override {
+        CUdeviceptr p = 0;
+        const int r = (int)reserve_(&p, size, align, 0, 0);
+        *va = (uint64_t)p;
+        return r;
+    }
+    int free_va(uint64_t va, size_t size) override { return (int)free_((CUdeviceptr)va, size); }
+    int create(uint64_t *handle, size_t size, int device) override {
+        CUmemAllocationProp prop = make_prop(device);
+        CUmemGenericAllocationHandle h = 0;
+        const int r = (int)create_(&h, size, &prop, 0);
+        *handle = (uint64_t)h;
+        return r;
+    }
+    int release(uint64_t handle) override { return (int)release_((CUmemGenericAllocationHandle)handle); }
+    int map(uint64_t va, size_t size, uint64_t handle) override {
+        return (int)map_((CUdeviceptr)va, size, 0, (CUmemGenericAllocationHandle)handle, 0);
+    }
+    int set_access(uint64_t va, size_t size, int device) override {
+        CUmemAccessDesc d;
+        std::memset(&d, 0, sizeof d);
+        d.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+        d.location.id = device;
+        d.flags = CU_MEM_ACCESS_FLAGS_PROT_READWRITE;
+        return (int)set_access_((CUdeviceptr)va, size, &d, 1);
+    }
+    int unmap(uint64_t va, size_t size) override { return (int)unmap_((CUdeviceptr)va, size); }
+    const char *name() const override { return "cuda"; }
+
+  private:
+    static CUmemAllocationProp make_prop(int device) {
+        CUmemAllocationProp prop;
+        std::memset(&prop, 0, sizeof prop);
+        prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
+        prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+        prop.location.id = device;
+        return prop;
+    }
+    template <typename F>
+    static bool get(const char *sym, F *fn, std::string *err) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        const cudaError_t e = cudaGetDriverEntryPoint(sym, &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+            if (err) *err = std::string("driver entry point not available: ") + sym;
+            return false;
+        }
+        *fn = reinterpret_cast<F>(p);
+        return true;
+    }
+    CUresult (*granularity_)(size_t *, const CUmemAllocationProp *, CUmemAllocationGranularity_flags) = nullptr;
+    CUresult (*reserve_)(CUdeviceptr *, size_t, size_t, CUdeviceptr, unsigned long long) = nullptr;
+    CUresult (*free_)(CUdeviceptr, size_t) = nullptr;
+    CUresult (*create_)(CUmemGenericAllocationHandle *, size_t, const CUmemAllocationProp *, unsigned long long) = nullptr;
+    CUresult (*release_)(CUmemGenericAllocationHandle) = nullptr;
+    CUresult (*map_)(CUdeviceptr, size_t, size_t, CUmemGenericAllocationHandle, unsigned long long) = nullptr;
+    CUresult (*set_access_)(CUdeviceptr, size_t, const CUmemAccessDesc *, size_t) = nullptr;
+    CUresult (*unmap_)(CUdeviceptr, size_t) = nullptr;
+};
+
+// ---- in-process fake: checks that the bookkeeping only issues legal sequences -------------------------------
+class FakeDriver final : public VmmDriver {
+  public:
+    explicit FakeDriver(uint32_t fail_nth_create) : fail_nth_(fail_nth_create) {}
+    int granularity(int, size_t *out) override {
+        *out = 2u << 20;
+        return 0;
+    }
+    int reserve(uint64_t *va, size_t size, size_t align) override {
+        if (align == 0) align = 2u << 20;
+        next_va_ = (next_va_ + align - 1) / align * align;
+        *va = next_va_;
+        ranges_[next_va_] = size;
+        next_va_ += size;
+        return 0;
+    }
+    int free_va(uint64_t va, size_t size) override {
+        auto it = ranges_.find(va);
+        if (it == ranges_.end() || it->second != size) return 1;
+        for (auto &m : maps_)
+            if (m.first >= va && m.first < va + size) return 1;  // still mapped
+        ranges_.erase(it);
+        return 0;
+    }
+    int create(uint64_t *handle, size_t size, int) override {
+        ++creates_;
+        if (fail_nth_ && creates_ == fail_nth_) return 2;  // out of memory
+        *handle = next_handle_++;
+        handles_[*handle] = size;
+        return 0;
+    }
+    int release(uint64_t handle) override { return handles_.erase(handle) ? 0 : 1; }
+    int map(uint64_t va, size_t size, uint64_t handle) override {
+        auto h = handles_.find(handle);
+        if (h == handles_.end() || h->second != size) return 1;
+        if (!inside_range(va, size) || overlaps(va, size)) return 1;
+        maps_[va] = {size, handle, false};
+        return 0;
+    }
+    int set_access(uint64_t va, size_t size, int) override {
+        uint64_t covered = va;
+        for (auto it = maps_.lower_bound(va); it != maps_.end() && it->first < va + size; ++it) {
+            if (it->first != covered) return 1;  // hole
+            it->second.accessible = true;
+            covered = it->first + it->second.size;
+        }
+        return covered == va + size ? 0 : 1;
+    }
+    int unmap(uint64_t va, size_t size) override {
+        auto it = maps_.find(va);
+        if (it == maps_.end() || it->second.size != size) return 1;
+        maps_.erase(it);
+        return 0;
+    }
+    const char *name() const override { return "fake"; }
+
+  private:
+    struct Mapping {
+        size_t size;
+        uint64_t handle;
+        bool accessible;
+    };
+    bool inside_range(uint64_t va, size_t size) const {
+        auto it = ranges_.upper_bound(va);
+        if (it == ranges_.begin()) return false;
+        --it;
+        return va + size <= it->first + it->second;
+    }
+    bool overlaps(uint64_t va, size_t size) const {
+        auto it = maps_.lower_bound(va);
+        if (it != maps_.end() && it->first < va + size) return true;
+        if (it != maps_.begin()) {
+            --it;
+            if (it->first + it->second.size > va) return true;
+        }
+        return false;
+    }
+    uint32_t fail_nth_, creates_ = 0;
+    uint64_t next_va_ = 0x700000000000ull, next_handle_ = 1;
+    std::map<uint64_t, size_t> ranges_, handles_;
+    std::map<uint64_t, Mapping> maps_;
+};
+
+}  // namespace
+
+std::unique_ptr<VmmDriver> make_cuda_driver(std::string *err) {
+    std::unique_ptr<CudaDriver> d(new CudaDriver());
+    if (!d->load(err)) return nullptr;
+    return d;
+}
+std::unique_ptr<VmmDriver> make_fake_driver(uint32_t fail_nth_create) {
+    return std::unique_ptr<VmmDriver>(new FakeDriver(fail_nth_create));
+}
+
+XTensor::XTensor(std::unique_ptr<VmmDriver> drv, int device, int32_t max_slots, int64_t max_seq_len, int64_t row_bytes)
+    : drv_(std::move(drv)), device_(device), max_seq_len_(max_seq_len), row_bytes_(row_bytes), slots_(max_slots) {}
+
+XTensor::~XTensor() { teardown(); }
+
+int XTensor::init_pool(int64_t phys_budget_bytes, int64_t page_bytes, bool lazy, std::string *err) {
+    size_t gran = 0;
+    if (drv_->granularity(device_, &gran) != 0 || gran == 0) {
+        *err = "cuMemGetAllocationGranularity failed";
+        return XLLM_ERR_CUDA;
+    }
+    if (page_bytes == 0) page_bytes = (int64_t)gran;
+    if (page_bytes % (int64_t)gran != 0) {
+        *err = "page_bytes must be a multiple of the device granularity (" + std::to_string(gran) + ")";
+        return XLLM_ERR_INVALID;
+    }
+    page_bytes_ = page_bytes;
+    lazy_ = lazy;
+    const int64_t block = (int64_t)XLLM_TILE_TOKENS * row_bytes_;
+    const int64_t blocks = (max_seq_len_ + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS;
+    va_bytes_ = (blocks * block + page_bytes_ - 1) / page_bytes_ * page_bytes_;
+    const int64_t n_pages = phys_budget_bytes / page_bytes_;
+    if (n_pages < 1) {
+        *err = "phys_budget_bytes is smaller than one page (" + std::to_string(page_bytes_) + " bytes)";
+        return XLLM_ERR_INVALID;
+    }
+    pages_.assign((size_t)n_pages, PageRecord());
+    free_.resize((size_t)n_pages);
+    for (int64_t i = 0; i < n_pages; ++i) free_[(size_t)i] = (int32_t)(n_pages - 1 - i);  // page 0 is popped first
+    if (!lazy_) {
+        for (int64_t i = 0; i < n_pages; ++i) {
+            if (drv_->create(&pages_[(size_t)i].handle, (size_t)page_bytes_, device_) != 0) {
+                *err = "cuMemCreate failed for page " + std::to_string(i) + " of " + std::to_string(n_pages) +
+                       " (budget exceeds free device memory?)";
+                return XLLM_ERR_OOM_PHYS;
+            }
+            pages_[(size_t)i].created = true;
+        }
+    }
+    return XLLM_OK;
+}
+
+int64_t XTensor::pages_for(int64_t tokens) const {
+    const int64_t blocks = (tokens + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS;
+    const int64_t bytes = blocks * XLLM_TILE_TOKENS * row_bytes_;
+    return (bytes + page_bytes_ - 1) / page_bytes_;
+}
+
+int64_t XTensor::mapped_tokens(int32_t s) const {
+    const int64_t blocks = ((int64_t)slots_[s].n_owned * page_bytes_) / ((int64_t)XLLM_TILE_TOKENS * row_bytes_);
+    return std::min(blocks * XLLM_TILE_TOKENS, (max_seq_len_ + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS * XLLM_TILE_TOKENS);
+}
+
+int XTensor::reserve(int64_t max_seq_len, int64_t expected_tokens, int32_t *slot_out, std::string *err) {
+    if (max_seq_len < 1 || max_seq_len > max_seq_len_ || expected_tokens < 0 || !slot_out) {
+        *err = "reserve: max_seq_len must be in [1, " + std::to_string(max_seq_len_) + "] and expected_tokens >= 0";
+        return XLLM_ERR_INVALID;
+    }
+    const int64_t need = pages_for(std::min(expected_tokens, max_seq_len_));
+    int32_t pick = -1, pick_fit = -1, pick_big = -1;
+    for (int32_t i = 0; i < (int32_t)slots_.size(); ++i) {
+        const SlotRecord &s = slots_[i];
+        if (s.live) continue;
+        if (pick < 0) pick = i;
+        const int64_t n = (int64_t)s.pages.size();
+        if (n == 0) continue;
+        if (n >= need && (pick_fit < 0 || n < (int64_t)slots_[pick_fit].pages.size())) pick_fit = i;
+        if (pick_big < 0 || n > (int64_t)slots_[pick_big].pages.size()) pick_big = i;
+    }
+    if (pick < 0) {
+        *err = "reserve: all " + std::to_string(slots_.size()) + " slots are live";
+        return XLLM_ERR_OOM_VA;
+    }
+    if (pick_fit >= 0) pick = pick_fit;
+    else if (pick_big >= 0 && need > 0) pick = pick_big;
+    SlotRecord &s = slots_[pick];
+    if (s.base == 0) {
+        if (drv_->reserve(&s.base, (size_t)va_bytes_, (size_t)page_bytes_) != 0 || s.base == 0) {
+            s.base = 0;
+            *err = "cuMemAddressReserve failed for " + std::to_string(va_bytes_) + " bytes";
+            return XLLM_ERR_OOM_VA;
+        }
+    }
+    s.live = true;
+    s.n_owned = 0;
+    s.kv_len = 0;
+    *slot_out = pick;
+    return XLLM_OK;
+}
+
+int XTensor::take_free_page(int32_t *page, std::string *err) {
+    const int32_t p = free_.back();
+    PageRecord &pr = pages_[p];
+    if (!pr.created) {
+        if (drv_->create(&pr.handle, (size_t)page_bytes_, device_) != 0) {
+            *err = "cuMemCreate failed for page " + std::to_string(p);
+            return XLLM_ERR_OOM_PHYS;
+        }
+        pr.created = true;
+    }
+    free_.pop_back();
+    pr.status = kAllocated;
+    *page = p;
+    return XLLM_OK;
+}
+
+int XTensor::unmap_page_at(SlotRecord &s, size_t pos) {
+    const double t0 = now_us();
+    const int r = drv_->unmap(s.base + pos * (uint64_t)page_bytes_, (size_t)page_bytes_);
+    unmap_us_ += now_us() - t0;
+    if (r == 0) ++unmapped_total_;
+    return r;
+}
+
+// Take one Reusable page away from another slot: released slots first, then live slots' reusable tails.
+bool XTensor::reclaim_one(int32_t needy, std::string *err, int *status) {
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int32_t i = 0; i < (int32_t)slots_.size(); ++i) {
+            SlotRecord &s = slots_[i];
+            if (i == needy || s.live != (pass == 1) || (int32_t)s.pages.size() <= s.n_owned) continue;
+            if (wait_idle) {
+                const int w = wait_idle(s);
+                if (w != 0) {
+                    *status = w;
+                    *err = "reclaim: slot " + std::to_string(i) + " still has work in flight";
+                    return false;
+                }
+            }
+            const int32_t p = s.pages.back();
+            if (unmap_page_at(s, s.pages.size() - 1) != 0) {
+                *status = XLLM_ERR_CUDA;
+                *err = "cuMemUnmap failed while reclaiming a reusable page";
+                return false;
+            }
+            s.pages.pop_back();
+            pages_[p].status = kFree;
+            pages_[p].owner = -1;
+            free_.push_back(p);
+            return true;
+        }
+    }
+    *status = XLLM_ERR_OOM_PHYS;
+    *err = "no reusable page left to reclaim";
+    return false;
+}
+
+int XTensor::map_pages(int32_t slot, int64_t min_tokens, std::string *err) {
+    if (!valid_slot(slot) || !slots_[slot].live || min_tokens < 0 || min_tokens > max_seq_len_) {
+        *err = "map_pages: slot must be live and 0 <= min_tokens <= " + std::to_string(max_seq_len_);
+        return XLLM_ERR_INVALID;
+    }
+    SlotRecord &s = slots_[slot];
+    const int64_t need = pages_for(min_tokens);
+    if (need <= s.n_owned) return XLLM_OK;
+    const int64_t promote = std::min<int64_t>(need, (int64_t)s.pages.size()) - s.n_owned;
+    const int64_t fresh = need - s.n_owned - promote;
+    int64_t reclaimable = 0;
+    for (int32_t i = 0; i < (int32_t)slots_.size(); ++i)
+        if (i != slot) reclaimable += (int64_t)slots_[i].pages.size() - slots_[i].n_owned;
+    if (fresh > (int64_t)free_.size() + reclaimable) {
+        *err = "map_pages: physical page pool exhausted (need " + std::to_string(fresh) + " more pages, " +
+               std::to_string(free_.size()) + " free, " + std::to_string(reclaimable) + " reclaimable)";
+        return XLLM_ERR_OOM_PHYS;
+    }
+    // 1. collect the fresh pages (Free -> Allocated), reclaiming reusable ones under pressure
+    std::vector<int32_t> got;
+    got.reserve((size_t)fresh);
+    int status = XLLM_OK;
+    for (int64_t i = 0; i < fresh && status == XLLM_OK; ++i) {
+        if (free_.empty() && !reclaim_one(slot, err, &status)) break;
+        int32_t p;
+        status = take_free_page(&p, err);
+        if (status == XLLM_OK) got.push_back(p);
+    }
+    // 2. map them at the next contiguous positions of the range and open access (Allocated -> Mapped)
+    size_t mapped_now = 0;
+    const size_t first_pos = s.pages.size();
+    if (status == XLLM_OK && !got.empty()) {
+        const double t0 = now_us();
+        for (; mapped_now < got.size(); ++mapped_now) {
+            const uint64_t va = s.base + (first_pos + mapped_now) * (uint64_t)page_bytes_;
+            if (drv_->map(va, (size_t)page_bytes_, pages_[got[mapped_now]].handle) != 0) {
+                status = XLLM_ERR_CUDA;
+                *err = "cuMemMap failed";
+                break;
+            }
+        }
+        if (status == XLLM_OK &&
+            drv_->set_access(s.base + first_pos * (uint64_t)page_bytes_, got.size() * (size_t)page_bytes_, device_) != 0) {
+            status = XLLM_ERR_CUDA;
+            *err = "cuMemSetAccess failed";
+        }
+        map_us_ += now_us() - t0;
+    }
+    if (status != XLLM_OK) {  // undo: nothing of this call stays mapped, the pages go back on the stack in order
+        for (size_t i = mapped_now; i-- > 0;) drv_->unmap(s.base + (first_pos + i) * (uint64_t)page_bytes_, (size_t)page_bytes_);
+        for (size_t i = got.size(); i-- > 0;) {
+            pages_[got[i]].status = kFree;
+            pages_[got[i]].owner = -1;
+            free_.push_back(got[i]);
+        }
+        return status;
+    }
+    // 3. commit
+    for (int64_t i = 0; i < promote; ++i) pages_[s.pages[(size_t)(s.n_owned + i)]].status = kMapped;
+    reused_total_ += promote;
+    s.n_owned += (int32_t)promote;
+    for (int32_t p : got) {
+        pages_[p].status = kMapped;
+        pages_[p].owner = slot;
+        s.pages.push_back(p);
+        ++s.n_owned;
+        ++mapped_total_;
+    }
+    return XLLM_OK;
+}
+
+int XTensor::release(int32_t slot, int32_t mode, std::string *err) {
+    if (!valid_slot(slot) || !slots_[slot].live || (mode != 0 && mode != 1)) {
+        *err = "release: slot must be live and mode 0 or 1";
+        return XLLM_ERR_INVALID;
+    }
+    SlotRecord &s = slots_[slot];
+    if (mode == 0) {
+        for (int32_t p : s.pages) pages_[p].status = kReusable;
+    } else {
+        if (wait_idle && !s.pages.empty()) {
+            const int w = wait_idle(s);
+            if (w != 0) {
+                *err = "release: slot still has work in flight";
+                return w;
+            }
+        }
+        for (size_t i = s.pages.size(); i-- > 0;) {
+            if (unmap_page_at(s, i) != 0) {
+                *err = "cuMemUnmap failed";
+                return XLLM_ERR_CUDA;
+            }
+            const int32_t p = s.pages[i];
+            s.pages.pop_back();
+            pages_[p].status = kFree;
+            pages_[p].owner = -1;
+            free_.push_back(p);
+        }
+    }
+    s.live = false;
+    s.n_owned = 0;
+    s.kv_len = 0;
+    return XLLM_OK;
+}
+
+void XTensor::teardown() {
+    if (!drv_) return;
+    for (SlotRecord &s : slots_) {
+        for (size_t i = s.pages.size(); i-- > 0;) drv_->unmap(s.base + i * (uint64_t)page_bytes_, (size_t)page_bytes_);
+        s.pages.clear();
+        if (s.base) drv_->free_va(s.base, (size_t)va_bytes_);
+        s.base = 0;
+        s.live = false;
+    }
+    for (PageRecord &p : pages_)
+        if (p.created) {
+            drv_->release(p.handle);
+            p.created = false;
+        }
+    pages_.clear();
+    free_.clear();
+}
+
+void XTensor::fill_stats(xllm_stats *st) const {
+    st->page_bytes = page_bytes_;
+    st->pages_total = (int64_t)pages_.size();
+    st->pages_free = st->pages_allocated = st->pages_mapped = st->pages_reusable = 0;
+    for (const PageRecord &p : pages_) {
+        switch (p.status) {
+            case kFree: ++st->pages_free; break;
+            case kAllocated: ++st->pages_allocated; break;
+            case kMapped: ++st->pages_mapped; break;
+            case kReusable: ++st->pages_reusable; break;
+        }
+    }
+    st->pages_mapped_total = mapped_total_;
+    st->pages_unmapped_total = unmapped_total_;
+    st->pages_reused_total = reused_total_;
+    st->map_host_us = map_us_;
+    st->unmap_host_us = unmap_us_;
+}
+
+}  // namespace xllm

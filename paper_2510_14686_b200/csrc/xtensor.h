@@ -1,0 +1,96 @@
+// xTensor mapper: physical page pool, per-slot virtual ranges, on-demand mapping, page reuse.
+#pragma once
+
+#include <cstdint>
+#include <functional>
+#include <memory>
+#include <string>
+#include <vector>
+
+#include "xllm_attn.h"
+
+namespace xllm {
+
+// Thin seam over the CUDA virtual-memory-management driver calls, so that the bookkeeping can also run
+// against an in-process fake (host tests, error injection).  Every method returns 0 on success.
+class VmmDriver {
+  public:
+    virtual ~VmmDriver() = default;
+    virtual int granularity(int device, size_t *out) = 0;
+    virtual int reserve(uint64_t *va, size_t size, size_t align) = 0;           // cuMemAddressReserve
+    virtual int free_va(uint64_t va, size_t size) = 0;                          // cuMemAddressFree
+    virtual int create(uint64_t *handle, size_t size, int device) = 0;          // cuMemCreate
+    virtual int release(uint64_t handle) = 0;                                   // cuMemRelease
+    virtual int map(uint64_t va, size_t size, uint64_t handle) = 0;             // cuMemMap
+    virtual int set_access(uint64_t va, size_t size, int device) = 0;           // cuMemSetAccess (read/write)
+    virtual int unmap(uint64_t va, size_t size) = 0;                            // cuMemUnmap
+    virtual const char *name() const = 0;
+};
+
+std::unique_ptr<VmmDriver> make_cuda_driver(std::string *err);       // resolved through the CUDA runtime
+std::unique_ptr<VmmDriver> make_fake_driver(uint32_t fail_nth_create);
+
+enum PageStatus : int8_t { kFree = 0, kAllocated = 1, kMapped = 2, kReusable = 3 };
+
+struct PageRecord {  // <PageID, Status, OwnerSession>; PageID is the index in the pool
+    PageStatus status = kFree;
+    int32_t owner = -1;  // slot id
+    uint64_t handle = 0;
+    bool created = false;
+};
+
+struct SlotRecord {
+    uint64_t base = 0;      // 0 until the slot id is first used
+    bool live = false;
+    std::vector<int32_t> pages;  // in virtual-address order
+    int32_t n_owned = 0;         // pages[:n_owned] are Mapped (owned by the live request), the rest Reusable
+    int64_t kv_len = 0;
+    uint64_t last_use = 0;       // sequence number of the last launch that touched the slot
+};
+
+class XTensor {
+  public:
+    XTensor(std::unique_ptr<VmmDriver> drv, int device, int32_t max_slots, int64_t max_seq_len, int64_t row_bytes);
+    ~XTensor();
+    // Returns an xllm_status; fills err on failure.
+    int init_pool(int64_t phys_budget_bytes, int64_t page_bytes, bool lazy, std::string *err);
+    int reserve(int64_t max_seq_len, int64_t expected_tokens, int32_t *slot_out, std::string *err);
+    int map_pages(int32_t slot, int64_t min_tokens, std::string *err);
+    int release(int32_t slot, int32_t mode, std::string *err);
+    void teardown();
+
+    int64_t pages_for(int64_t tokens) const;
+    int64_t mapped_tokens(int32_t slot) const;
+    bool valid_slot(int32_t slot) const { return slot >= 0 && slot < (int32_t)slots_.size(); }
+    SlotRecord &slot(int32_t s) { return slots_[s]; }
+    const SlotRecord &slot(int32_t s) const { return slots_[s]; }
+    const std::vector<PageRecord> &pages() const { return pages_; }
+    int64_t page_bytes() const { return page_bytes_; }
+    int64_t va_bytes() const { return va_bytes_; }
+    int64_t row_bytes() const { return row_bytes_; }
+    int64_t max_seq_len() const { return max_seq_len_; }
+    void fill_stats(xllm_stats *st) const;
+    VmmDriver &driver() { return *drv_; }
+    int device() const { return device_; }
+
+    // Called before pages of a slot are unmapped; must return 0 once no work in flight uses the slot,
+    // or XLLM_ERR_BUSY to refuse.
+    std::function<int(const SlotRecord &)> wait_idle;
+
+  private:
+    int take_free_page(int32_t *page, std::string *err);
+    bool reclaim_one(int32_t needy, std::string *err, int *status);
+    int unmap_page_at(SlotRecord &s, size_t pos);
+
+    std::unique_ptr<VmmDriver> drv_;
+    int device_;
+    int64_t max_seq_len_, row_bytes_, page_bytes_ = 0, va_bytes_ = 0;
+    bool lazy_ = false;
+    std::vector<PageRecord> pages_;
+    std::vector<int32_t> free_;  // stack: back() is popped first
+    std::vector<SlotRecord> slots_;
+    int64_t mapped_total_ = 0, unmapped_total_ = 0, reused_total_ = 0;
+    double map_us_ = 0.0, unmap_us_ = 0.0;
+};
+
+}  // namespace xllm

@@ -1,0 +1,89 @@
+"""GPU: the ten-step continuous-batching scenario (on-demand mapping, append, mixed decode/verify, draft
+rollback, release with and without unmap, slot take-over), every step compared with the oracle and the page
+counters compared with the page-pool model."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import PagePoolModel
+from paper_2510_14686_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+def run_scenario(binding, n_requests, steps, max_len, n_pages):
+    import gpu_harness as gh
+
+    sc = wl.PagedScenario(n_requests=n_requests, steps=steps, max_len=max_len)
+    s = sc.shape
+    page = 2 << 20
+    max_seq = max_len + 64
+    ctx = binding.Context(s.n_q_heads, s.n_kv_heads, s.head_dim, n_requests, max_seq, n_pages * page, max_q_len=4)
+    model = PagePoolModel(n_pages, page, s.row_bytes, binding.TILE_TOKENS, n_requests, max_seq)
+    slot_of = {}
+
+    def admit(r, k, v):
+        n = k.shape[0]
+        sl, ml = ctx.kv_reserve(expected_tokens=n + 4), model.reserve(n + 4)
+        assert sl == ml
+        ctx.kv_map_pages(sl, n)
+        assert model.map_pages(ml, n) == 0
+        if n:
+            ctx.kv_append([sl], [n], gh.dev_bits(k), gh.dev_bits(v))
+        slot_of[r] = sl
+
+    for r in range(n_requests):
+        admit(r, sc.k[r], sc.v[r])
+    worst = (0.0, 0.0)
+    for plan in sc.plans():
+        n = n_requests
+        slots = [slot_of[r] for r in range(n)]
+        for r in range(n):                                      # (1) map on demand
+            need = sc.cached_len(r) + int(plan.q_lens[r])
+            ctx.kv_map_pages(slots[r], need)
+            assert model.map_pages(slots[r], need) == 0
+        ctx.kv_append(slots, plan.q_lens, gh.dev_bits(np.concatenate(plan.new_k)), gh.dev_bits(np.concatenate(plan.new_v)))  # (2)
+        reqs = [wl.Request(int(plan.q_lens[r]), sc.cached_len(r) + int(plan.q_lens[r]), plan.q[r],
+                           np.concatenate([sc.k[r], plan.new_k[r]]), np.concatenate([sc.v[r], plan.new_v[r]])) for r in range(n)]
+        batch = wl.Batch(s, reqs)
+        out, lse = gh.run_attention(ctx, batch, slots, use_decode=False)   # (3) one call, mixed q_lens
+        mx, mean = gh.assert_parity(out, lse, *gh.oracle_batch(batch))     # (4)
+        worst = (max(worst[0], mx), max(worst[1], mean))
+        for r in range(n):                                      # (5) roll back rejected drafts
+            if plan.q_lens[r] == 4:
+                ctx.kv_set_len(slots[r], reqs[r].kv_len - (3 - int(plan.accepted[r])))
+        for r in plan.finished:                                 # (6) finish + admit
+            ctx.kv_release(slots[r], plan.release_mode[r])
+            assert model.release(slots[r], plan.release_mode[r]) == 0
+        for r in plan.finished:
+            admit(r, plan.admitted[r].k, plan.admitted[r].v)
+        st = ctx.get_stats()
+        c = model.counts()
+        assert (st.pages_free, st.pages_mapped, st.pages_reusable) == (c["free"], c["mapped"], c["reusable"])
+        assert (st.pages_mapped_total, st.pages_unmapped_total, st.pages_reused_total) == (
+            model.pages_mapped_total, model.pages_unmapped_total, model.pages_reused_total)
+    # after the script the library's view of every live sequence equals the host copy
+    for r in range(n_requests):
+        assert ctx.kv_slot_info(slot_of[r]).kv_len == sc.cached_len(r)
+    st = ctx.get_stats()
+    ctx.shutdown()
+    return worst, st
+
+
+def test_small_scenario_under_memory_pressure(binding):
+    worst, st = run_scenario(binding, n_requests=24, steps=6, max_len=3000, n_pages=40)
+    assert st.pages_reused_total > 0
+
+
+def test_full_scenario_256_requests_ten_steps(binding):
+    worst, st = run_scenario(binding, n_requests=256, steps=10, max_len=32768, n_pages=420)
+    print(f"paged: worst max-abs {worst[0]:.2e} mean-abs {worst[1]:.2e}; mapped {st.pages_mapped_total} "
+          f"unmapped {st.pages_unmapped_total} reused {st.pages_reused_total}; map {st.map_host_us:.0f} us unmap {st.unmap_host_us:.0f} us")
+    assert st.pages_reused_total > 0 and st.pages_unmapped_total > 0

@@ -1,0 +1,138 @@
+"""xTensor bookkeeping of the library (host-only context, fake driver) against the page-pool model."""
+import numpy as np
+import pytest
+
+from oracle import PagePoolModel
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import build
+
+    build.build()
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+PAGE = 2 << 20
+
+
+def make(binding, n_pages=16, slots=6, hq=32, hkv=8, d=128, max_len=8192, **kw):
+    ctx = binding.Context(hq, hkv, d, slots, max_len, n_pages * PAGE, flags=binding.FLAG_HOST_ONLY | kw.pop("flags", 0), **kw)
+    model = PagePoolModel(n_pages, PAGE, 2 * hkv * d * 2, binding.TILE_TOKENS, slots, max_len)
+    return ctx, model
+
+
+def same_state(ctx, model):
+    st = ctx.get_stats()
+    c = model.counts()
+    assert (st.pages_free, st.pages_allocated, st.pages_mapped, st.pages_reusable) == (c["free"], c["allocated"], c["mapped"], c["reusable"])
+    assert (st.pages_mapped_total, st.pages_unmapped_total, st.pages_reused_total) == (
+        model.pages_mapped_total, model.pages_unmapped_total, model.pages_reused_total)
+    for i, s in model.slots.items():
+        info = ctx.kv_slot_info(i)
+        assert (info.live, info.pages_in_range, info.pages_owned) == (int(s.live), len(s.pages), s.n_owned)
+        assert info.mapped_tokens == model.mapped_tokens(i)
+        for pos, p in enumerate(s.pages):    # Eq. 2 through the library's table: same page ids in the same order
+            assert ctx.kv_page_of(i, pos * PAGE + 12345) == (pos, p, 12345)
+        if len(s.pages) * PAGE < info.va_bytes:
+            with pytest.raises(ctx_error(ctx)) as e:
+                ctx.kv_page_of(i, len(s.pages) * PAGE)
+            assert e.value.status == -4
+
+
+def ctx_error(ctx):
+    from paper_2510_14686_b200.binding import XllmError
+
+    return XllmError
+
+
+def test_random_walk_matches_model(binding):
+    rng = np.random.default_rng(11)
+    ctx, model = make(binding)
+    live = set()
+    for step in range(600):
+        op = int(rng.integers(0, 3))
+        if op == 0 and len(live) < 6:
+            hint = int(rng.integers(0, 3000))
+            a, b = ctx.kv_reserve(expected_tokens=hint), model.reserve(hint)
+            assert a == b
+            live.add(a)
+        elif op == 1 and live:
+            s = int(rng.choice(sorted(live)))
+            t = int(rng.integers(1, 5000))
+            want = model.map_pages(s, t)
+            if want == 0:
+                ctx.kv_map_pages(s, t)
+            else:
+                with pytest.raises(binding.XllmError) as e:
+                    ctx.kv_map_pages(s, t)
+                assert e.value.status == want
+        elif op == 2 and live:
+            s = int(rng.choice(sorted(live)))
+            mode = int(rng.integers(0, 2))
+            ctx.kv_release(s, mode)
+            assert model.release(s, mode) == 0
+            live.discard(s)
+        if step % 20 == 0:
+            same_state(ctx, model)
+    same_state(ctx, model)
+    model.check_invariants()
+    ctx.shutdown()
+
+
+def test_slot_ranges_are_disjoint_and_sized_for_max_seq_len(binding):
+    ctx, _ = make(binding, max_len=5000)
+    slots = [ctx.kv_reserve() for _ in range(6)]
+    infos = [ctx.kv_slot_info(s) for s in slots]
+    need = -(-5000 // 64) * 64 * infos[0].row_bytes
+    for i in infos:
+        assert i.base % PAGE == 0 and i.va_bytes >= need and i.va_bytes % PAGE == 0 and i.row_bytes == 4096
+    spans = sorted((i.base, i.base + i.va_bytes) for i in infos)
+    assert all(a[1] <= b[0] for a, b in zip(spans[:-1], spans[1:]))
+    with pytest.raises(binding.XllmError) as e:
+        ctx.kv_reserve()
+    assert e.value.status == binding.ERR_OOM_VA
+    # the range survives release and is handed to the next request with the same id
+    ctx.kv_release(slots[2], 1)
+    assert ctx.kv_reserve() == slots[2] and ctx.kv_slot_info(slots[2]).base == infos[2].base
+
+
+def test_set_len_and_argument_errors(binding):
+    ctx, _ = make(binding)
+    s = ctx.kv_reserve()
+    ctx.kv_map_pages(s, 700)      # 2 pages = 1024 tokens
+    ctx.kv_set_len(s, 1024)
+    ctx.kv_set_len(s, 3)
+    assert ctx.kv_slot_info(s).kv_len == 3
+    for bad in (lambda: ctx.kv_set_len(s, 1025), lambda: ctx.kv_set_len(s, -1), lambda: ctx.kv_set_len(5, 0),
+                lambda: ctx.kv_map_pages(s, 8193), lambda: ctx.kv_map_pages(3, 10), lambda: ctx.kv_release(s, 7),
+                lambda: ctx.kv_reserve(max_seq_len=8193)):
+        with pytest.raises(binding.XllmError) as e:
+            bad()
+        assert e.value.status == binding.ERR_INVALID
+    assert ctx.kv_slot_info(s).kv_len == 3 and ctx.kv_slot_info(s).pages_owned == 2
+
+
+def test_lazy_pool_driver_failure_leaves_state_unchanged(binding):
+    # the fake driver refuses its 3rd page creation: the call fails as OOM_PHYS and nothing stays mapped
+    ctx, model = make(binding, flags=binding.FLAG_LAZY_PAGES, fault_inject=3)
+    s = ctx.kv_reserve()
+    ctx.kv_map_pages(s, 1000)                       # pages 0, 1
+    before = ctx.get_stats().as_dict()
+    with pytest.raises(binding.XllmError) as e:
+        ctx.kv_map_pages(s, 2500)                   # needs pages 2 (creation fails), 3, 4
+    assert e.value.status == binding.ERR_OOM_PHYS
+    after = ctx.get_stats().as_dict()
+    for k in ("pages_free", "pages_mapped", "pages_allocated", "pages_reusable", "pages_mapped_total"):
+        assert before[k] == after[k]
+    assert ctx.kv_slot_info(s).pages_owned == 2
+    ctx.kv_map_pages(s, 2500)                       # the next attempt succeeds and continues the range in order
+    assert [ctx.kv_page_of(s, i * PAGE)[1] for i in range(5)] == [0, 1, 2, 3, 4]
+
+
+def test_eager_pool_creation_failure_is_reported(binding):
+    with pytest.raises(binding.XllmError) as e:
+        make(binding, fault_inject=5)
+    assert e.value.status == binding.ERR_OOM_PHYS

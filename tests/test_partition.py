@@ -1,0 +1,104 @@
+"""Host work partition: every visible key of every (request, KV head, row group) is covered exactly once,
+CTA loads are near equal, pieces of a split unit are consecutive and never start where a row sees no key."""
+import numpy as np
+import pytest
+
+from paper_2510_14686_b200 import workloads as wl
+
+T = 64
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import build
+
+    build.build()
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+def check_plan(binding, kv, ql, hq, hkv, n_ctas):
+    items, cta, n_units, n_parts = binding.plan_partition(kv, ql, hq, hkv, n_ctas)
+    G = hq // hkv
+    assert cta[0] == 0 and cta[-1] == len(items) and np.all(np.diff(cta) >= 0)
+    cover = {}
+    partial_ids = []
+    loads = np.zeros(n_ctas, np.int64)
+    for c in range(n_ctas):
+        for it in items[cta[c]:cta[c + 1]]:
+            # cost axis of the planner: 4 per tile plus 3 for starting a unit
+            loads[c] += 4 * (it.tile_end - it.tile_begin) + (3 if it.tile_begin == 0 else 0)
+            key = (it.req, it.kv_head, it.q_tok0, it.g0)
+            q_len = 1 if ql is None else int(ql[it.req])
+            vis_last = int(kv[it.req]) - q_len + it.q_tok0 + it.n_q_tok
+            vis_first = int(kv[it.req]) - q_len + it.q_tok0 + 1
+            n_tiles = -(-vis_last // T)
+            assert 0 <= it.tile_begin < it.tile_end <= n_tiles
+            assert it.n_q_tok * it.n_g <= 16 and it.n_q_tok >= 1 and it.n_g >= 1
+            assert it.g0 + it.n_g <= G and it.q_tok0 + it.n_q_tok <= q_len
+            assert it.tile_begin * T < vis_first, "a piece must hold a key visible to its first row"
+            cover.setdefault(key, []).append((it.tile_begin, it.tile_end, n_tiles, it.partial_idx, it.unit))
+            if it.partial_idx >= 0:
+                partial_ids.append(it.partial_idx)
+    assert sorted(partial_ids) == list(range(n_parts))
+    assert len(cover) == n_units
+    # rows: every (request, query token, query head) belongs to exactly one unit
+    rows = set()
+    for (req, h, t0, g0), pieces in cover.items():
+        pieces.sort()
+        assert pieces[0][0] == 0 and pieces[-1][1] == pieces[0][2]
+        for a, b in zip(pieces[:-1], pieces[1:]):
+            assert a[1] == b[0]
+        if len(pieces) == 1:
+            assert pieces[0][3] == -1
+        else:
+            ids = [p[3] for p in pieces]
+            assert ids == list(range(ids[0], ids[0] + len(ids))) and ids[0] >= 0
+        assert len({p[4] for p in pieces}) == 1
+    for it in items:
+        for t in range(it.q_tok0, it.q_tok0 + it.n_q_tok):
+            for g in range(it.g0, it.g0 + it.n_g):
+                rows.add((it.req, t, it.kv_head * G + g))
+    total_rows = sum((1 if ql is None else int(x)) for x in (ql if ql is not None else kv)) * hq if ql is not None else len(kv) * hq
+    assert len(rows) == total_rows
+    return items, loads, n_parts
+
+
+@pytest.mark.parametrize("name", ["tiny", "decode", "verify", "longctx", "paged"])
+def test_named_workloads(binding, name):
+    kv, ql = wl.draw_lengths(name)
+    s = wl.SHAPES[name]
+    items, loads, n_parts = check_plan(binding, kv, ql, s.n_q_heads, s.n_kv_heads, 148)
+    total = loads.sum()
+    if name != "tiny":
+        # near-equal cost per CTA (slack: the no-sliver rule may move a cut by a few tiles)
+        assert loads.max() - total / 148 <= 4 * 6, (loads.max(), total / 148)
+        assert n_parts <= 2 * 148
+
+
+def test_small_and_odd_cases(binding):
+    check_plan(binding, np.array([1]), None, 4, 1, 148)
+    check_plan(binding, np.array([64, 65, 63, 1, 128]), np.array([1, 2, 3, 1, 4], np.int32), 8, 2, 7)
+    check_plan(binding, np.array([5000]), np.array([4], np.int32), 28, 4, 148)     # G = 7: two row groups of 2 tokens
+    check_plan(binding, np.array([300, 9]), np.array([3, 3], np.int32), 32, 1, 16)  # G = 32 > 16: head sub-groups
+    check_plan(binding, np.array([131072]), None, 8, 8, 148)
+    check_plan(binding, np.array([4, 4, 4]), np.array([4, 4, 4], np.int32), 4, 4, 1)
+
+
+def test_random_cases(binding):
+    rng = np.random.default_rng(3)
+    for _ in range(60):
+        n = int(rng.integers(1, 40))
+        hkv = int(rng.choice([1, 2, 4, 8]))
+        g = int(rng.choice([1, 2, 4, 5, 7, 8, 16]))
+        ql = rng.integers(1, 5, n).astype(np.int32)
+        kv = np.maximum(ql, (rng.pareto(1.0, n) * 200).astype(np.int64) + 1)
+        check_plan(binding, kv, ql, hkv * g, hkv, int(rng.choice([1, 3, 16, 148])))
+
+
+def test_rejects_bad_input(binding):
+    with pytest.raises(binding.XllmError):
+        binding.plan_partition([3], [4], 4, 1, 8)    # kv_len < q_len
+    with pytest.raises(binding.XllmError):
+        binding.plan_partition([3], [1], 5, 2, 8)    # heads not divisible

@@ -167,6 +167,10 @@ xllm_status xllm_kv_page_of(const xllm_ctx *ctx, int32_t slot, int64_t byte_offs
 xllm_status xllm_debug_read_slot(xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int64_t nbytes, void *host_dst);
 xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_offset, int64_t nbytes, void *host_dst);
 
+/* Inspection: per-CTA cycle counters of the last attention launch (16 words per CTA; layout documented beside the
+ * kernel).  Only collected when the process was started with XLLM_TRACE=1 in the environment; else UNSUPPORTED. */
+xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max_words, int32_t *n_words_out);
+
 /* ---- KV writes ("write_kvcache": only a start address and offsets, no block table) ---------------------- */
 
 /* Append n_new[i] tokens to slot slots[i] for i < n_req: rows k_new / v_new (device, bf16,

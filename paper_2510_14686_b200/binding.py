@@ -88,6 +88,7 @@ EXPORTS = {
     "xllm_kv_page_of": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, _i32p, _i32p, _i64p]),
     "xllm_debug_read_slot": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
     "xllm_debug_read_page": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
+    "xllm_debug_read_trace": (ctypes.c_int32, [_ctxp, ctypes.POINTER(ctypes.c_uint64), ctypes.c_int32, _i32p]),
     "xllm_kv_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i32p, _vp, _vp, _vp]),
     "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
     "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _vp, _vp, _vp, ctypes.c_float, _vp]),
@@ -223,6 +224,12 @@ class Context:
         buf = np.empty(nbytes, np.uint8)
         self._check(_lib.xllm_debug_read_page(self._ctx, page_id, byte_offset, nbytes, buf.ctypes.data))
         return buf
+
+    def debug_read_trace(self) -> np.ndarray:
+        buf = np.zeros(160 * 16, np.uint64)
+        n = ctypes.c_int32()
+        self._check(_lib.xllm_debug_read_trace(self._ctx, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)), len(buf), ctypes.byref(n)))
+        return buf[:n.value].reshape(-1, 16)
 
     # -- KV writes --
     def kv_append(self, slots, n_new, k_new, v_new, stream=None):

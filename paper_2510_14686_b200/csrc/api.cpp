@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <memory>
 #include <string>
@@ -48,6 +49,7 @@ struct xllm_ctx {
     cudaStream_t last_stream = nullptr;
 
     float *d_part_o = nullptr, *d_part_lse = nullptr;
+    unsigned long long *d_trace = nullptr;  // per-CTA cycle counters, only when XLLM_TRACE is set in the environment
     int32_t max_partials = 0, max_items = 0;
     int32_t *h_error = nullptr, *d_error = nullptr;  // mapped pinned word written by kernels whose waits expired
 
@@ -228,24 +230,27 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     int idx;
     int e = acquire_stage(ctx, &idx);
     if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
-    // layout of the staged blob
+    // staged blob: resolved items, then combine descriptors
     const size_t off_items = 0;
-    const size_t off_cta = align_up(off_items + sizeof(xllm_work_item) * (size_t)n_items, 16);
-    const size_t off_reqs = align_up(off_cta + sizeof(int32_t) * (size_t)(ctx->sm_count + 1), 16);
-    const size_t off_comb = align_up(off_reqs + sizeof(ReqDesc) * (size_t)n_req, 16);
+    const size_t off_comb = align_up(off_items + sizeof(DevItem) * (size_t)n_items, 16);
     const size_t total = align_up(off_comb + sizeof(CombineDesc) * combine.size(), 16);
     if (total > ctx->stage_bytes) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
     char *h = ctx->h_stage[idx];
-    std::memcpy(h + off_items, ctx->items.data(), sizeof(xllm_work_item) * (size_t)n_items);
-    std::memcpy(h + off_cta, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
-    ReqDesc *rd = reinterpret_cast<ReqDesc *>(h + off_reqs);
-    for (int32_t i = 0; i < n_req; ++i) {
-        SlotRecord &s = ctx->xt->slot(slots[i]);
-        rd[i].base = s.base;
-        rd[i].kv_len = (int32_t)s.kv_len;
-        rd[i].q_len = q_lens ? q_lens[i] : 1;
-        rd[i].q_row0 = q_row0[(size_t)i];
-        rd[i].pad = 0;
+    DevItem *di = reinterpret_cast<DevItem *>(h + off_items);
+    const int64_t head_tile = head_tile_bytes(ctx->cfg.head_dim);
+    for (int32_t i = 0; i < n_items; ++i) {
+        const xllm_work_item &w = ctx->items[(size_t)i];
+        const SlotRecord &s = ctx->xt->slot(slots[w.req]);
+        const int32_t ql = q_lens ? q_lens[w.req] : 1;
+        di[i].kv = s.base + (uint64_t)(w.kv_head * head_tile);
+        di[i].q_row = q_row0[(size_t)w.req] + w.q_tok0;
+        di[i].partial_idx = w.partial_idx;
+        di[i].tile_begin = w.tile_begin;
+        di[i].tile_end = w.tile_end;
+        di[i].kv_end = (int32_t)s.kv_len - ql + w.q_tok0 + w.n_q_tok;
+        di[i].head0 = (int16_t)(w.kv_head * G + w.g0);
+        di[i].n_q_tok = (uint8_t)w.n_q_tok;
+        di[i].n_g = (uint8_t)w.n_g;
     }
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
 
@@ -255,20 +260,20 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     if (e) return cuda_fail(ctx, "staging the work list", e);
 
     AttnLaunch al{};
-    al.items = reinterpret_cast<const xllm_work_item *>(d + off_items);
-    al.cta_begin = reinterpret_cast<const int32_t *>(d + off_cta);
-    al.reqs = reinterpret_cast<const ReqDesc *>(d + off_reqs);
+    al.items = reinterpret_cast<const DevItem *>(d + off_items);
     al.q = q;
     al.out = out;
     al.lse_out = lse_out;
     al.part_o = ctx->d_part_o;
     al.part_lse = ctx->d_part_lse;
     al.error_flag = ctx->d_error;
+    al.trace = ctx->d_trace;
     al.n_q_heads = ctx->cfg.n_q_heads;
     al.n_kv_heads = ctx->cfg.n_kv_heads;
     al.head_dim = ctx->cfg.head_dim;
     al.scale_log2 = scale * 1.4426950408889634f;
     al.n_ctas = ctx->sm_count;
+    std::memcpy(al.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
     time_begin(ctx, 0, stream);
     e = launch_attention(al, stream);
     time_end(ctx, stream);
@@ -340,7 +345,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         cudaGetDeviceProperties(&prop, cfg->device);
         if (prop.major != 10) return bad(XLLM_ERR_UNSUPPORTED, "kernels are built for sm_100a only; device is sm_" +
                                                                   std::to_string(prop.major) + std::to_string(prop.minor));
-        ctx->sm_count = prop.multiProcessorCount;
+        ctx->sm_count = std::min<int>(prop.multiProcessorCount, kMaxCtas);
         std::string derr;
         drv = make_cuda_driver(&derr);
         if (!drv) return bad(XLLM_ERR_CUDA, derr);
@@ -361,10 +366,9 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
                                            : cfg->max_q_len * ((G + kMaxRows - 1) / kMaxRows);
     ctx->max_items = cfg->max_slots * cfg->n_kv_heads * groups + ctx->sm_count + 1;
     ctx->max_partials = 2 * ctx->sm_count + 2;
-    ctx->stage_bytes = align_up(sizeof(xllm_work_item) * (size_t)ctx->max_items, 16) +
-                       align_up(sizeof(int32_t) * (size_t)(ctx->sm_count + 1), 16) +
-                       align_up(std::max(sizeof(ReqDesc), sizeof(AppendDesc)) * (size_t)cfg->max_slots, 16) +
-                       align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16) + 64;
+    ctx->stage_bytes = std::max(align_up(sizeof(DevItem) * (size_t)ctx->max_items, 16) +
+                                    align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16),
+                                align_up(sizeof(AppendDesc) * (size_t)cfg->max_slots, 16)) + 64;
     if (!ctx->host_only) {
         cudaError_t e = cudaSuccess;
         for (int i = 0; i < kRing && e == cudaSuccess; ++i) {
@@ -378,6 +382,11 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         if (e == cudaSuccess) {
             *ctx->h_error = 0;
             e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&ctx->d_error), ctx->h_error, 0);
+        }
+        if (e == cudaSuccess && std::getenv("XLLM_TRACE")) {
+            const size_t tb = sizeof(unsigned long long) * (size_t)ctx->sm_count * kTraceWords;
+            e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_trace), tb);
+            if (e == cudaSuccess) e = cudaMemset(ctx->d_trace, 0, tb);
         }
         if (e == cudaSuccess) e = (cudaError_t)configure_kernels(cfg->head_dim);
         if (e != cudaSuccess) {
@@ -407,6 +416,7 @@ xllm_status xllm_shutdown(xllm_ctx *ctx) {
         }
         if (ctx->d_part_o) cudaFree(ctx->d_part_o);
         if (ctx->d_part_lse) cudaFree(ctx->d_part_lse);
+        if (ctx->d_trace) cudaFree(ctx->d_trace);
         if (ctx->h_error) cudaFreeHost(ctx->h_error);
         for (TimedLaunch &t : ctx->timed) {
             cudaEventDestroy(t.start);
@@ -538,6 +548,17 @@ xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_of
     return st;
 }
 
+xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max_words, int32_t *n_words_out) {
+    if (!ctx || !host_dst || !n_words_out) return XLLM_ERR_INVALID;
+    if (!ctx->d_trace) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_trace: start the process with XLLM_TRACE=1 to collect a trace");
+    const int32_t n = std::min(max_words, ctx->sm_count * kTraceWords);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(host_dst, ctx->d_trace, sizeof(uint64_t) * (size_t)n, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, "debug_read_trace", (int)e);
+    *n_words_out = n;
+    return XLLM_OK;
+}
+
 xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new, const void *k_new,
                            const void *v_new, void *cuda_stream) {
     if (!ctx) return XLLM_ERR_INVALID;
@@ -567,8 +588,9 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     int e = acquire_stage(ctx, &idx);
     if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
     AppendDesc *ad = reinterpret_cast<AppendDesc *>(ctx->h_stage[idx]);
-    int32_t row0 = 0, n_desc = 0;
+    int32_t row0 = 0, n_desc = 0, max_new = 0;
     for (int32_t i = 0; i < n_req; ++i) {
+        max_new = std::max(max_new, n_new[i]);
         if (n_new[i] == 0) continue;
         const SlotRecord &s = ctx->xt->slot(slots[i]);
         ad[n_desc++] = {s.base, (int32_t)s.kv_len, row0, n_new[i], 0};
@@ -578,7 +600,7 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     e = (int)cudaMemcpyAsync(ctx->d_stage[idx], ad, sizeof(AppendDesc) * (size_t)n_desc, cudaMemcpyHostToDevice, stream);
     if (e) return cuda_fail(ctx, "staging the append list", e);
     time_begin(ctx, 2, stream);
-    e = launch_append(reinterpret_cast<const AppendDesc *>(ctx->d_stage[idx]), n_desc, (int32_t)rows, k_new, v_new,
+    e = launch_append(reinterpret_cast<const AppendDesc *>(ctx->d_stage[idx]), n_desc, max_new, k_new, v_new,
                       ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);
     time_end(ctx, stream);
     if (e) return cuda_fail(ctx, "launching the append kernel", e);

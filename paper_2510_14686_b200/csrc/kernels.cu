@@ -9,12 +9,14 @@
 // softmax state (running max, sum, fp32 output accumulator) for all query rows of the GQA group
 // (rows = heads of the group x query tokens <= 16), so every K/V byte is fetched from HBM once for
 // all of them.  Q.K^T and P.V run on mma.sync m16n8k16 bf16 (the work is HBM bound: ~rows flop/byte).
-// At the end of an item the eight per-warp states are merged through shared memory and either the
-// final bf16 output or an fp32 partial (+ log2-domain LSE) is written.  The speculative-verification
+// At the end of an item each consumer warp drops its state into shared memory and moves on; warps 9-11
+// (epilogue) merge the eight states and write either the final bf16 output or an fp32 partial (+ log2-domain
+// LSE) while the consumers already work on the next item.  The speculative-verification
 // causal mask only touches the tiles that hold the newest q_len tokens.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 
 #include "xllm_internal.h"
@@ -24,30 +26,21 @@ namespace {
 
 constexpr int T = XLLM_TILE_TOKENS;
 constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;
+constexpr int kProducerWarp = kConsumerWarps;          // warp 8
+constexpr int kEpilogueWarp0 = kConsumerWarps + 1;     // warps 9..11
+constexpr int kEpilogueWarps = 3;
+constexpr int kEpilogueThreads = kEpilogueWarps * 32;
+constexpr int kThreads = (kConsumerWarps + 1 + kEpilogueWarps) * 32;  // 384
 constexpr int kItemBatch = 64;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // a bounded wait gives up after 2 s
-
-struct __align__(16) RItem {  // work item resolved against the request table, kept in shared memory
-    const char *kv;           // head tile of tile block 0
-    const char *q;            // first query row of the group
-    char *out;                // bf16 final rows or fp32 partial rows
-    float *lse;               // may be null (final) / partial lse
-    int32_t tile_begin, tile_end;
-    int32_t kv_end;           // keys visible to the group's last row; tokens beyond are neither fetched nor used
-    int32_t row_limit0;       // keys visible to the group's first query token
-    int32_t n_q_tok, n_g;
-    int32_t is_partial;
-    int32_t pad;
-};
-static_assert(sizeof(RItem) == 64, "RItem layout");
 
 template <int D>
 struct Cfg {
     static constexpr int kPanels = D / 64;
     static constexpr int kHeadTile = 2 * kPanels * kPanelBytes;      // K + V of one head, 64 tokens
-    static constexpr int kStages = 4 * (128 / D);
+    static constexpr int kHalfTile = kPanels * kPanelBytes;          // K or V of one head, 64 tokens
+    static constexpr int kStages = 4 * (128 / D);                    // tiles of ring capacity
+    static constexpr int kHalfStages = 2 * kStages;                  // K and V halves are acquired and released separately
     static constexpr int kQPitch = D * 2 + 16;                       // bytes, padded against bank conflicts
     static constexpr int kOPitch = D + 8;                            // floats
     static constexpr int kOffStages = 0;
@@ -56,8 +49,8 @@ struct Cfg {
     static constexpr int kOffMergeL = kOffMergeM + kConsumerWarps * kMaxRows * 4;
     static constexpr int kOffQ = kOffMergeL + kConsumerWarps * kMaxRows * 4;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
-    static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(RItem);
-    static constexpr int kNumBars = 2 * kStages + 4;
+    static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(DevItem);
+    static constexpr int kNumBars = 2 * kHalfStages + 6;
     static constexpr int kOffFlags = kOffBars + kNumBars * 8;
     static constexpr int kSmemBytes = kOffFlags + 16;
 };
@@ -135,193 +128,212 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
 
 // ---- one 16-token slice of a tile, all query rows ---------------------------------------------------------
-template <int D, bool MASK>
-__device__ __forceinline__ void slice_compute(uint32_t stage, int wslice, int lane, const uint32_t (&qf)[D / 16][4],
-                                              float (&o)[D / 8][4], float (&m)[2], float (&l)[2], float scale_log2,
-                                              int tok_base, int limit_lo, int limit_hi, int kv_end) {
-    constexpr int kPanels = D / 64;
+// Phase 1 (needs the K half of the tile): scores, mask, online-softmax update; returns the bf16 weights as an MMA
+// A fragment.  HALF: the item has at most 8 rows, so rows 8..15 of the MMA tile are padding and are skipped.
+template <int D, bool MASK, bool HALF>
+__device__ __forceinline__ void slice_scores(uint32_t kstage, int wslice, int lane, const uint32_t (&qf)[D / 16][4],
+                                             float (&o)[D / 8][4], float (&m)[2], float (&l)[2], float scale_log2,
+                                             int tok_base, int limit_lo, int limit_hi, uint32_t (&pa)[4]) {
     const int swz = lane & 7;
+    // two accumulation chains per 8-token block (even / odd k-steps) to shorten the dependent MMA chain
     float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float s2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     {
         const int r = wslice * 16 + (lane & 7) + ((lane >> 4) << 3);
         const int csel = (lane >> 3) & 1;
-        const uint32_t row_addr = stage + r * 128;
+        const uint32_t row_addr = kstage + r * 128;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-            const int cg = 2 * ks + csel;
-            uint32_t b0, b1, b2, b3;
+        for (int ks = 0; ks < D / 16; ks += 2) {
+            uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+            const int cg = 2 * ks + csel, cg2 = cg + 2;
             ldsm_x4(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
+            ldsm_x4(c0, c1, c2, c3, row_addr + (cg2 >> 3) * kPanelBytes + (((cg2 & 7) ^ swz) << 4));
             mma_bf16(s[0], qf[ks], b0, b1);
             mma_bf16(s[1], qf[ks], b2, b3);
+            mma_bf16(s2[0], qf[ks + 1], c0, c1);
+            mma_bf16(s2[1], qf[ks + 1], c2, c3);
         }
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[nt][e] += s2[nt][e];
     }
     const int q4 = lane & 3;
     if (MASK) {
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
+            for (int e = 0; e < (HALF ? 2 : 4); ++e) {
                 const int tok = tok_base + nt * 8 + 2 * q4 + (e & 1);
                 if (tok >= ((e < 2) ? limit_lo : limit_hi)) s[nt][e] = -INFINITY;
             }
     }
     float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-    float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    const float mn0 = fmaxf(m[0], mx0 * scale_log2), mn1 = fmaxf(m[1], mx1 * scale_log2);
-    const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-    const float a0 = exp2f(m[0] - ms0), a1 = exp2f(m[1] - ms1);
+    const float mn0 = fmaxf(m[0], mx0 * scale_log2);
+    const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0;
+    const float a0 = exp2f(m[0] - ms0);
     m[0] = mn0;
-    m[1] = mn1;
+    float ms1 = 0.f, a1 = 1.f;
+    if (!HALF) {
+        float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        const float mn1 = fmaxf(m[1], mx1 * scale_log2);
+        ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        a1 = exp2f(m[1] - ms1);
+        m[1] = mn1;
+    }
     float p[2][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
         p[nt][0] = exp2f(fmaf(s[nt][0], scale_log2, -ms0));
         p[nt][1] = exp2f(fmaf(s[nt][1], scale_log2, -ms0));
-        p[nt][2] = exp2f(fmaf(s[nt][2], scale_log2, -ms1));
-        p[nt][3] = exp2f(fmaf(s[nt][3], scale_log2, -ms1));
+        p[nt][2] = HALF ? 0.f : exp2f(fmaf(s[nt][2], scale_log2, -ms1));
+        p[nt][3] = HALF ? 0.f : exp2f(fmaf(s[nt][3], scale_log2, -ms1));
     }
     l[0] = l[0] * a0 + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
-    l[1] = l[1] * a1 + (p[0][2] + p[0][3] + p[1][2] + p[1][3]);
+    if (!HALF) l[1] = l[1] * a1 + (p[0][2] + p[0][3] + p[1][2] + p[1][3]);
+    if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {  // the running maximum moved: rescale the accumulator
 #pragma unroll
-    for (int nt = 0; nt < D / 8; ++nt) {
-        o[nt][0] *= a0;
-        o[nt][1] *= a0;
-        o[nt][2] *= a1;
-        o[nt][3] *= a1;
+        for (int nt = 0; nt < D / 8; ++nt) {
+            o[nt][0] *= a0;
+            o[nt][1] *= a0;
+            if (!HALF) {
+                o[nt][2] *= a1;
+                o[nt][3] *= a1;
+            }
+        }
     }
-    const uint32_t pa[4] = {pack_bf16(p[0][0], p[0][1]), pack_bf16(p[0][2], p[0][3]), pack_bf16(p[1][0], p[1][1]),
-                            pack_bf16(p[1][2], p[1][3])};
+    pa[0] = pack_bf16(p[0][0], p[0][1]);
+    pa[1] = HALF ? 0u : pack_bf16(p[0][2], p[0][3]);
+    pa[2] = pack_bf16(p[1][0], p[1][1]);
+    pa[3] = HALF ? 0u : pack_bf16(p[1][2], p[1][3]);
+}
+
+// Phase 2 (needs the V half): O += P . V for the slice's 16 tokens.
+template <int D, bool MASK>
+__device__ __forceinline__ void slice_pv(uint32_t vstage, int wslice, int lane, const uint32_t (&pa)[4], float (&o)[D / 8][4],
+                                         int tok_base, int kv_end) {
+    const int swz = lane & 7, q4 = lane & 3;
     uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
     if (MASK) {  // V rows never written by append may hold anything: force them to zero (0 * NaN would poison O)
         const int t0 = tok_base + 2 * q4;
         vmask0 = (t0 < kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < kv_end ? 0xffff0000u : 0u);
         vmask1 = (t0 + 8 < kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < kv_end ? 0xffff0000u : 0u);
     }
-    {
-        const int r = wslice * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-        const int csel = lane >> 4;
-        const uint32_t row_addr = stage + kPanels * kPanelBytes + r * 128;
+    const int r = wslice * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+    const int csel = lane >> 4;
+    const uint32_t row_addr = vstage + r * 128;
 #pragma unroll
-        for (int n2 = 0; n2 < D / 16; ++n2) {
-            const int cg = 2 * n2 + csel;
-            uint32_t b0, b1, b2, b3;
-            ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
-            if (MASK) {
-                b0 &= vmask0;
-                b1 &= vmask1;
-                b2 &= vmask0;
-                b3 &= vmask1;
-            }
-            mma_bf16(o[2 * n2], pa, b0, b1);
-            mma_bf16(o[2 * n2 + 1], pa, b2, b3);
+    for (int n2 = 0; n2 < D / 16; ++n2) {
+        const int cg = 2 * n2 + csel;
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
+        if (MASK) {
+            b0 &= vmask0;
+            b1 &= vmask1;
+            b2 &= vmask0;
+            b3 &= vmask1;
         }
+        mma_bf16(o[2 * n2], pa, b0, b1);
+        mma_bf16(o[2 * n2 + 1], pa, b2, b3);
     }
 }
 
 // ---- split-KV attention ---------------------------------------------------------------------------------
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const AttnLaunch p) {
+// Warp roles: 0-7 consumers (two groups of four taking alternate tiles), 8 producer (bulk copies), 9-11 epilogue
+// (merge the eight per-warp states of a finished item and write its result while the consumers go on).
+template <int D, bool TRACE>
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnLaunch p) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem_base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    RItem *ritems = reinterpret_cast<RItem *>(smem + C::kOffItems);
+    const DevItem *sitems = reinterpret_cast<const DevItem *>(smem + C::kOffItems);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::kOffFlags);
-    const uint32_t bar_full = smem_base + C::kOffBars;               // [kStages]
-    const uint32_t bar_empty = bar_full + C::kStages * 8;             // [kStages]
-    const uint32_t bar_qfull = bar_empty + C::kStages * 8;            // [2]
-    const uint32_t bar_qempty = bar_qfull + 16;                       // [2]
+    const uint32_t bar_full = smem_base + C::kOffBars;               // [kHalfStages] K or V half of a tile landed
+    const uint32_t bar_empty = bar_full + C::kHalfStages * 8;         // [kHalfStages] ... consumed (4 warps)
+    const uint32_t bar_qfull = bar_empty + C::kHalfStages * 8;        // [2] query rows landed
+    const uint32_t bar_qempty = bar_qfull + 16;                       // [2] query rows loaded to registers (8 warps)
+    const uint32_t bar_mfull = bar_qempty + 16;                       // per-warp states of an item written (8 warps)
+    const uint32_t bar_mempty = bar_mfull + 8;                        // ... and read by the epilogue (3 warps)
+    const unsigned long long t_start = TRACE ? clock64() : 0ull;
+    const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
 
+    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
     if (tid == 0) {
-        for (int s = 0; s < C::kStages; ++s) {
+        for (int s = 0; s < C::kHalfStages; ++s) {
             mbar_init(bar_full + s * 8, 1);
-            mbar_init(bar_empty + s * 8, 4);  // the four warps of the consuming group
+            mbar_init(bar_empty + s * 8, 4);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_qfull + b * 8, 1);
             mbar_init(bar_qempty + b * 8, kConsumerWarps);
         }
+        mbar_init(bar_mfull, kConsumerWarps);
+        mbar_init(bar_mempty, kEpilogueWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
 
-    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
-    const int G = p.n_q_heads / p.n_kv_heads;
     const int64_t tile_block = (int64_t)p.n_kv_heads * C::kHeadTile;
     uint32_t fill = 0;      // tiles issued / consumed so far by this CTA (same sequence in every warp)
     uint32_t item_seq = 0;  // items started so far
+    unsigned long long tr_wait_full = 0, tr_compute = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0,
+                       tr_epi = 0;
 
     for (int batch_lo = item_lo; batch_lo < item_hi; batch_lo += kItemBatch) {
         const int nb = min(kItemBatch, item_hi - batch_lo);
         if (batch_lo != item_lo) __syncthreads();  // everyone is done with the previous batch's records
-        for (int i = tid; i < nb; i += kThreads) {
-            const xllm_work_item w = p.items[batch_lo + i];
-            const ReqDesc rq = p.reqs[w.req];
-            RItem r;
-            r.kv = reinterpret_cast<const char *>(rq.base) + (int64_t)w.kv_head * C::kHeadTile;
-            const int64_t row0 = rq.q_row0 + w.q_tok0;
-            const int head0 = w.kv_head * G + w.g0;
-            r.q = static_cast<const char *>(p.q) + (row0 * p.n_q_heads + head0) * (int64_t)(D * 2);
-            r.is_partial = w.partial_idx >= 0;
-            if (r.is_partial) {
-                r.out = reinterpret_cast<char *>(p.part_o + (int64_t)w.partial_idx * kMaxRows * D);
-                r.lse = p.part_lse + (int64_t)w.partial_idx * kMaxRows;
-            } else {
-                r.out = static_cast<char *>(p.out) + (row0 * p.n_q_heads + head0) * (int64_t)(D * 2);
-                r.lse = p.lse_out ? p.lse_out + row0 * p.n_q_heads + head0 : nullptr;
-            }
-            r.tile_begin = w.tile_begin;
-            r.tile_end = w.tile_end;
-            r.row_limit0 = rq.kv_len - rq.q_len + w.q_tok0 + 1;
-            r.kv_end = r.row_limit0 + w.n_q_tok - 1;
-            r.n_q_tok = w.n_q_tok;
-            r.n_g = w.n_g;
-            r.pad = 0;
-            ritems[i] = r;
-        }
+        for (int i = tid; i < nb * 2; i += kThreads)   // 32-byte records moved as 16-byte halves
+            reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
         __syncthreads();
 
-        if (warp == kConsumerWarps) {
+        if (warp == kProducerWarp) {
             // ================= producer =================
             if (lane == 0) {
                 for (int i = 0; i < nb; ++i) {
-                    const RItem &it = ritems[i];
+                    const DevItem it = sitems[i];
                     const int n_rows = it.n_q_tok * it.n_g;
                     const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
                     if (mbar_wait(bar_qempty + qb * 8, qph ^ 1, abort_flag, p.error_flag, 1)) {
                         mbar_expect_tx(bar_qfull + qb * 8, n_rows * D * 2);
                         const uint32_t qdst = smem_base + C::kOffQ + qb * (kMaxRows * C::kQPitch);
+                        const char *qsrc = static_cast<const char *>(p.q) + ((int64_t)it.q_row * p.n_q_heads + it.head0) * (D * 2);
                         for (int t = 0; t < it.n_q_tok; ++t)
                             for (int g = 0; g < it.n_g; ++g)
-                                bulk_g2s(qdst + (t * it.n_g + g) * C::kQPitch,
-                                         it.q + ((int64_t)t * p.n_q_heads + g) * (D * 2), D * 2, bar_qfull + qb * 8);
+                                bulk_g2s(qdst + (t * it.n_g + g) * C::kQPitch, qsrc + ((int64_t)t * p.n_q_heads + g) * (D * 2),
+                                         D * 2, bar_qfull + qb * 8);
                     }
+                    const char *kv = reinterpret_cast<const char *>(it.kv);
                     for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
                         const uint32_t s = fill % C::kStages, ph = (fill / C::kStages) & 1;
-                        if (!mbar_wait(bar_empty + s * 8, ph ^ 1, abort_flag, p.error_flag, 2)) continue;
                         const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);
                         const uint32_t bytes = rows * 128;
-                        mbar_expect_tx(bar_full + s * 8, 2 * C::kPanels * bytes);
-                        const char *src = it.kv + (int64_t)tile * tile_block;
-                        const uint32_t dst = smem_base + C::kOffStages + s * C::kHeadTile;
+                        const char *src = kv + (int64_t)tile * tile_block;
 #pragma unroll
-                        for (int pn = 0; pn < 2 * C::kPanels; ++pn)
-                            bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, bytes, bar_full + s * 8);
+                        for (int half = 0; half < 2; ++half) {  // K half, then V half
+                            const uint32_t hs = 2 * s + half;
+                            const unsigned long long t0 = TRACE ? clock64() : 0ull;
+                            if (!mbar_wait(bar_empty + hs * 8, ph ^ 1, abort_flag, p.error_flag, 2)) continue;
+                            if (TRACE) tr_wait_empty += clock64() - t0;
+                            mbar_expect_tx(bar_full + hs * 8, C::kPanels * bytes);
+                            const uint32_t dst = smem_base + C::kOffStages + hs * C::kHalfTile;
+#pragma unroll
+                            for (int pn = 0; pn < C::kPanels; ++pn)
+                                bulk_g2s(dst + pn * kPanelBytes, src + (half * C::kPanels + pn) * kPanelBytes, bytes, bar_full + hs * 8);
+                        }
                     }
                 }
             } else {
-                for (int i = 0; i < nb; ++i) fill += ritems[i].tile_end - ritems[i].tile_begin;
+                for (int i = 0; i < nb; ++i) fill += sitems[i].tile_end - sitems[i].tile_begin;
             }
             fill = __shfl_sync(0xffffffffu, fill, 0);
-        } else {
+        } else if (warp < kConsumerWarps) {
             // ================= consumers =================
             const int group = warp >> 2, wslice = warp & 3;
             const int g8 = lane >> 2, q4 = lane & 3;
@@ -329,11 +341,14 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const AttnLaunch
             float *merge_m = reinterpret_cast<float *>(smem + C::kOffMergeM);
             float *merge_l = reinterpret_cast<float *>(smem + C::kOffMergeL);
             for (int i = 0; i < nb; ++i) {
-                const RItem it = ritems[i];
+                const DevItem it = sitems[i];
                 const int n_rows = it.n_q_tok * it.n_g;
-                const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
+                const int row_limit0 = it.kv_end - it.n_q_tok + 1;
+                const uint32_t seq = item_seq + i, qb = seq & 1, qph = (seq >> 1) & 1;
                 uint32_t qf[D / 16][4];
+                unsigned long long t0 = TRACE ? clock64() : 0ull;
                 bool live = mbar_wait(bar_qfull + qb * 8, qph, abort_flag, p.error_flag, 3);
+                if (TRACE) tr_wait_q += clock64() - t0;
                 {
                     const uint32_t qsrc = smem_base + C::kOffQ + qb * (kMaxRows * C::kQPitch) +
                                           ((lane & 7) + (((lane >> 3) & 1) << 3)) * C::kQPitch + ((lane >> 4) << 4);
@@ -347,8 +362,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const AttnLaunch
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_qempty + qb * 8);
 
-                const int limit_lo = (g8 < n_rows) ? it.row_limit0 + g8 / it.n_g : 0;
-                const int limit_hi = (g8 + 8 < n_rows) ? it.row_limit0 + (g8 + 8) / it.n_g : 0;
+                const int limit_lo = (g8 < n_rows) ? row_limit0 + g8 / it.n_g : 0;
+                const int limit_hi = (g8 + 8 < n_rows) ? row_limit0 + (g8 + 8) / it.n_g : 0;
+                const bool half = n_rows <= 8;
                 float o[D / 8][4];
 #pragma unroll
                 for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
@@ -357,114 +373,168 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const AttnLaunch
                 for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
                     if ((int)(fill & 1) != group) continue;
                     const uint32_t s = fill % C::kStages, ph = (fill / C::kStages) & 1;
-                    live = mbar_wait(bar_full + s * 8, ph, abort_flag, p.error_flag, 4) && live;
+                    const uint32_t bk = bar_full + (2 * s) * 8, bv = bk + 8;
+                    const uint32_t kstage = smem_base + C::kOffStages + (2 * s) * C::kHalfTile, vstage = kstage + C::kHalfTile;
                     const int tok_base = tile * T + wslice * 16;
-                    if (live && tok_base < it.kv_end) {
-                        const uint32_t stage = smem_base + C::kOffStages + s * C::kHeadTile;
-                        if (tile * T + T > it.row_limit0)
-                            slice_compute<D, true>(stage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo,
-                                                   limit_hi, it.kv_end);
-                        else
-                            slice_compute<D, false>(stage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo,
-                                                    limit_hi, it.kv_end);
+                    const bool work = tok_base < it.kv_end;
+                    const bool mask = tile * T + T > row_limit0;
+                    uint32_t pa[4];
+                    t0 = TRACE ? clock64() : 0ull;
+                    live = mbar_wait(bk, ph, abort_flag, p.error_flag, 4) && live;
+                    if (TRACE) {
+                        const unsigned long long t1 = clock64();
+                        tr_wait_full += t1 - t0;
+                        if (!tr_first) tr_first = t1 - t_start;
+                        t0 = t1;
+                    }
+                    if (live && work) {
+                        if (half) {
+                            if (mask) slice_scores<D, true, true>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
+                            else slice_scores<D, false, true>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
+                        } else {
+                            if (mask) slice_scores<D, true, false>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
+                            else slice_scores<D, false, false>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
+                        }
                     }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty + s * 8);
+                    if (lane == 0) mbar_arrive(bar_empty + (2 * s) * 8);      // K half is free again
+                    if (TRACE) {
+                        const unsigned long long t1 = clock64();
+                        tr_compute += t1 - t0;
+                        t0 = t1;
+                    }
+                    live = mbar_wait(bv, ph, abort_flag, p.error_flag, 7) && live;
+                    if (TRACE) {
+                        const unsigned long long t1 = clock64();
+                        tr_wait_full += t1 - t0;
+                        t0 = t1;
+                    }
+                    if (live && work) {
+                        if (mask) slice_pv<D, true>(vstage, wslice, lane, pa, o, tok_base, it.kv_end);
+                        else slice_pv<D, false>(vstage, wslice, lane, pa, o, tok_base, it.kv_end);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty + (2 * s + 1) * 8);  // V half is free again
+                    if (TRACE) tr_compute += clock64() - t0;
                 }
 
-                // ---- merge the eight per-warp states and write the item's result ----
+                // ---- hand the warp's state to the epilogue warps and go on with the next item ----
+                t0 = TRACE ? clock64() : 0ull;
                 l[0] += __shfl_xor_sync(0xffffffffu, l[0], 1);
                 l[1] += __shfl_xor_sync(0xffffffffu, l[1], 1);
                 l[0] += __shfl_xor_sync(0xffffffffu, l[0], 2);
                 l[1] += __shfl_xor_sync(0xffffffffu, l[1], 2);
-                consumer_bar();  // the previous item's merge buffers have been read
+                mbar_wait(bar_mempty, (seq + 1) & 1, abort_flag, p.error_flag, 5);  // previous item's states were read
                 if (q4 == 0) {
                     merge_m[warp * kMaxRows + g8] = m[0];
-                    merge_m[warp * kMaxRows + g8 + 8] = m[1];
                     merge_l[warp * kMaxRows + g8] = l[0];
-                    merge_l[warp * kMaxRows + g8 + 8] = l[1];
+                    if (!half) {
+                        merge_m[warp * kMaxRows + g8 + 8] = m[1];
+                        merge_l[warp * kMaxRows + g8 + 8] = l[1];
+                    }
                 }
                 {
+                    // always written: a warp that saw no visible key holds exact zeros, which the epilogue weighs by 0
                     float *dst = merge_o + (warp * kMaxRows + g8) * C::kOPitch + 2 * q4;
-                    if (m[0] != -INFINITY) {
 #pragma unroll
-                        for (int nt = 0; nt < D / 8; ++nt)
-                            *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
-                    }
-                    if (m[1] != -INFINITY) {
+                    for (int nt = 0; nt < D / 8; ++nt)
+                        *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+                    if (!half) {
 #pragma unroll
                         for (int nt = 0; nt < D / 8; ++nt)
                             *reinterpret_cast<float2 *>(dst + 8 * C::kOPitch + nt * 8) = make_float2(o[nt][2], o[nt][3]);
                     }
                 }
-                consumer_bar();
-                {
-                    constexpr int kPer = D / 16;  // output columns per thread
-                    const int row = tid >> 4, d0 = (tid & 15) * kPer;
-                    if (row < n_rows) {
-                        float M = -INFINITY;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_mfull);
+                if (TRACE) tr_switch += clock64() - t0;
+            }
+        } else {
+            // ================= epilogue =================
+            const int et = tid - kEpilogueWarp0 * 32;
+            const float *merge_o = reinterpret_cast<const float *>(smem + C::kOffMergeO);
+            const float *merge_m = reinterpret_cast<const float *>(smem + C::kOffMergeM);
+            const float *merge_l = reinterpret_cast<const float *>(smem + C::kOffMergeL);
+            constexpr int kC4 = D / 4;  // float4 columns per row
+            for (int i = 0; i < nb; ++i) {
+                const DevItem it = sitems[i];
+                const int n_rows = it.n_q_tok * it.n_g;
+                const uint32_t seq = item_seq + i;
+                const bool live = mbar_wait(bar_mfull, seq & 1, abort_flag, p.error_flag, 6);
+                const unsigned long long t0 = TRACE ? clock64() : 0ull;
+                for (int idx = et; live && idx < n_rows * kC4; idx += kEpilogueThreads) {
+                    const int row = idx / kC4, c4 = idx - row * kC4;
+                    float mw[kConsumerWarps];
+                    float M = -INFINITY;
 #pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_m[w * kMaxRows + row]);
-                        float acc[kPer];
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        mw[w] = merge_m[w * kMaxRows + row];
+                        M = fmaxf(M, mw[w]);
+                    }
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float L = 0.f;
+                    {
+                        const float Ms = (M == -INFINITY) ? 0.f : M;
 #pragma unroll
-                        for (int j = 0; j < kPer; ++j) acc[j] = 0.f;
-                        float L = 0.f;
-                        if (M != -INFINITY) {
-#pragma unroll
-                            for (int w = 0; w < kConsumerWarps; ++w) {
-                                const float mw = merge_m[w * kMaxRows + row];
-                                if (mw == -INFINITY) continue;
-                                const float wgt = exp2f(mw - M);
-                                L += wgt * merge_l[w * kMaxRows + row];
-                                const float *src = merge_o + (w * kMaxRows + row) * C::kOPitch + d0;
-#pragma unroll
-                                for (int j = 0; j < kPer; j += 4) {
-                                    const float4 v = *reinterpret_cast<const float4 *>(src + j);
-                                    acc[j] += wgt * v.x;
-                                    acc[j + 1] += wgt * v.y;
-                                    acc[j + 2] += wgt * v.z;
-                                    acc[j + 3] += wgt * v.w;
-                                }
-                            }
-                        }
-                        const float inv = (L > 0.f) ? 1.f / L : 0.f;
-                        const float lse2 = (L > 0.f) ? M + log2f(L) : -INFINITY;
-                        if (it.is_partial) {
-                            float *dst = reinterpret_cast<float *>(it.out) + row * D + d0;
-#pragma unroll
-                            for (int j = 0; j < kPer; j += 4)
-                                *reinterpret_cast<float4 *>(dst + j) =
-                                    make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv);
-                            if ((tid & 15) == 0) it.lse[row] = lse2;
-                        } else {
-                            const int ti = row / it.n_g, gi = row - ti * it.n_g;
-                            const int64_t off = (int64_t)ti * p.n_q_heads + gi;
-                            uint32_t packed[kPer / 2];
-#pragma unroll
-                            for (int j = 0; j < kPer; j += 2) packed[j / 2] = pack_bf16(acc[j] * inv, acc[j + 1] * inv);
-                            char *dst = it.out + off * (D * 2) + d0 * 2;
-                            if constexpr (kPer == 8)
-                                *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                            else
-                                *reinterpret_cast<uint2 *>(dst) = make_uint2(packed[0], packed[1]);
-                            if ((tid & 15) == 0 && it.lse) it.lse[off] = lse2 * 0.69314718055994531f;
+                        for (int w = 0; w < kConsumerWarps; ++w) {
+                            const float wgt = exp2f(mw[w] - Ms);  // 0 for a warp that saw no visible key (its O row is all zeros)
+                            L += wgt * merge_l[w * kMaxRows + row];
+                            const float4 v = *reinterpret_cast<const float4 *>(merge_o + (w * kMaxRows + row) * C::kOPitch + c4 * 4);
+                            acc.x += wgt * v.x;
+                            acc.y += wgt * v.y;
+                            acc.z += wgt * v.z;
+                            acc.w += wgt * v.w;
                         }
                     }
+                    const float inv = (L > 0.f) ? 1.f / L : 0.f;
+                    const float lse2 = (L > 0.f) ? M + log2f(L) : -INFINITY;
+                    if (it.partial_idx >= 0) {
+                        float *dst = p.part_o + ((int64_t)it.partial_idx * kMaxRows + row) * D + c4 * 4;
+                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                        if (c4 == 0) p.part_lse[(int64_t)it.partial_idx * kMaxRows + row] = lse2;
+                    } else {
+                        const int ti = row / it.n_g, gi = row - ti * it.n_g;
+                        const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
+                        *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
+                            make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                        if (c4 == 0 && p.lse_out) p.lse_out[off] = lse2 * 0.69314718055994531f;
+                    }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_mempty);
+                if (TRACE) tr_epi += clock64() - t0;
             }
+            for (int i = 0; i < nb; ++i) fill += sitems[i].tile_end - sitems[i].tile_begin;
         }
         item_seq += nb;
+    }
+
+    if (TRACE && lane == 0 && (warp == 0 || warp == 4 || warp == kProducerWarp || warp == kEpilogueWarp0)) {
+        unsigned long long *tr = p.trace + (int64_t)blockIdx.x * kTraceWords;
+        const unsigned long long total = clock64() - t_start;
+        if (warp == 0) {
+            tr[0] = total; tr[1] = tr_first; tr[2] = tr_wait_full; tr[3] = tr_compute; tr[4] = tr_wait_q; tr[5] = tr_switch;
+            tr[6] = (unsigned long long)(item_hi - item_lo); tr[7] = fill;
+            tr[15] = globaltimer_ns() - g_start;
+        } else if (warp == 4) {
+            tr[8] = tr_wait_full; tr[9] = tr_compute; tr[10] = tr_switch;
+        } else if (warp == kProducerWarp) {
+            tr[11] = tr_wait_empty; tr[12] = total;
+        } else {
+            tr[13] = tr_epi; tr[14] = total;
+        }
     }
 
     // Leave only when none of this CTA's bulk copies can still be in flight.  On the normal path every issued
     // copy was waited for by its consumers; after an abort the producer lane drains what it issued (bounded).
     __syncthreads();
-    if (*abort_flag && warp == kConsumerWarps && lane == 0) {
+    if (*abort_flag && warp == kProducerWarp && lane == 0) {
         const unsigned long long t0 = globaltimer_ns();
         for (uint32_t back = 0; back < (uint32_t)C::kStages && back < fill; ++back) {
             const uint32_t f = fill - 1 - back, s = f % C::kStages, ph = (f / C::kStages) & 1;
-            while (!mbar_try_wait(bar_full + s * 8, ph) && globaltimer_ns() - t0 < kWaitLimitNs) {
-            }
+            for (uint32_t hs = 2 * s; hs < 2 * s + 2; ++hs)
+                while (!mbar_try_wait(bar_full + hs * 8, ph) && globaltimer_ns() - t0 < kWaitLimitNs) {
+                }
         }
     }
 }
@@ -506,26 +576,21 @@ __device__ __forceinline__ int64_t slot_chunk_offset(int64_t pos, int h, int whi
            (int64_t)which * (panels * kPanelBytes) + (c >> 3) * kPanelBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
 }
 
-__global__ void append_kernel(const AppendDesc *__restrict__ descs, int n_req, int n_rows, const uint4 *__restrict__ k_new,
+__global__ void append_kernel(const AppendDesc *__restrict__ descs, const uint4 *__restrict__ k_new,
                               const uint4 *__restrict__ v_new, int n_kv_heads, int D) {
-    const int cpr = D / 8;  // chunks per head row
-    const int64_t per_tensor = (int64_t)n_rows * n_kv_heads * cpr;
-    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (id >= 2 * per_tensor) return;
-    const int which = id >= per_tensor;
-    const int64_t rem = id - which * per_tensor;
-    const int c = (int)(rem % cpr);
-    const int h = (int)((rem / cpr) % n_kv_heads);
-    const int row = (int)(rem / ((int64_t)cpr * n_kv_heads));
-    int lo = 0, hi = n_req - 1;  // last request whose first row is <= row
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (descs[mid].row0 <= row) lo = mid; else hi = mid - 1;
+    const AppendDesc d = descs[blockIdx.y];
+    const int cpr = D / 8;                       // chunks per head row
+    const int row_chunks = n_kv_heads * cpr;     // chunks per token of one tensor
+    const int64_t per_tensor = (int64_t)d.n_new * row_chunks;
+    for (int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; id < 2 * per_tensor; id += (int64_t)gridDim.x * blockDim.x) {
+        const int which = id >= per_tensor;
+        const int64_t rem = id - which * per_tensor;
+        const int c = (int)(rem % cpr);
+        const int h = (int)((rem / cpr) % n_kv_heads);
+        const int row = (int)(rem / row_chunks);
+        const uint4 val = (which ? v_new : k_new)[(int64_t)d.row0 * row_chunks + rem];
+        *reinterpret_cast<uint4 *>(d.base + slot_chunk_offset((int64_t)d.pos0 + row, h, which, c, n_kv_heads, D)) = val;
     }
-    const AppendDesc d = descs[lo];
-    const int64_t pos = (int64_t)d.pos0 + (row - d.row0);
-    const uint4 val = (which ? v_new : k_new)[rem];
-    *reinterpret_cast<uint4 *>(d.base + slot_chunk_offset(pos, h, which, c, n_kv_heads, D)) = val;
 }
 
 __global__ void gather_kernel(uint64_t base, int64_t first_token, int64_t n_tokens, uint4 *__restrict__ k_out,
@@ -550,19 +615,27 @@ int attention_smem_bytes(int32_t head_dim) { return head_dim == 128 ? Cfg<128>::
 
 int configure_kernels(int32_t head_dim) {
     cudaError_t e;
-    if (head_dim == 128)
-        e = cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
-    else
-        e = cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+    if (head_dim == 128) {
+        e = cudaFuncSetAttribute(attention_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+    } else {
+        e = cudaFuncSetAttribute(attention_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+    }
     return (int)e;
 }
 
 int launch_attention(const AttnLaunch &p, void *stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (p.head_dim == 128)
-        attention_kernel<128><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
-    else
-        attention_kernel<64><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+    if (p.head_dim == 128) {
+        if (p.trace) attention_kernel<128, true><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
+        else attention_kernel<128, false><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
+    } else {
+        if (p.trace) attention_kernel<64, true><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+        else attention_kernel<64, false><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+    }
     return (int)cudaGetLastError();
 }
 
@@ -576,13 +649,14 @@ int launch_combine(const CombineLaunch &p, void *stream) {
     return (int)cudaGetLastError();
 }
 
-int launch_append(const AppendDesc *descs, int32_t n_req, int32_t n_rows, const void *k_new, const void *v_new,
+int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *k_new, const void *v_new,
                   int32_t n_kv_heads, int32_t head_dim, void *stream) {
-    const int64_t total = 2ll * n_rows * n_kv_heads * (head_dim / 8);
+    const int64_t per_req = 2ll * max_new * n_kv_heads * (head_dim / 8);  // chunks of the largest request
     const int threads = 256;
-    const int64_t blocks = (total + threads - 1) / threads;
-    append_kernel<<<(unsigned)blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
-        descs, n_req, n_rows, static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), n_kv_heads, head_dim);
+    const int64_t bx = std::min<int64_t>((per_req + threads - 1) / threads, 4096);
+    dim3 grid((unsigned)bx, (unsigned)n_req);
+    append_kernel<<<grid, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        descs, static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), n_kv_heads, head_dim);
     return (int)cudaGetLastError();
 }
 

@@ -32,13 +32,18 @@ inline int64_t head_tile_bytes(int32_t head_dim) { return 2ll * (head_dim / 64) 
 inline int64_t tile_block_bytes(int32_t n_kv_heads, int32_t head_dim) { return n_kv_heads * head_tile_bytes(head_dim); }
 
 // ---- device-side records ------------------------------------------------------------------------------
-struct ReqDesc {            // one per request of an attention call
-    uint64_t base;          // slot range start
-    int32_t kv_len;
-    int32_t q_len;
-    int32_t q_row0;         // first row of the request in q / out
-    int32_t pad;
+constexpr int32_t kMaxCtas = 160;  // upper bound on the persistent grid (B200: 148 SMs)
+
+struct DevItem {            // one work item, resolved on the host against the slot table (32 bytes)
+    uint64_t kv;            // address of the item's KV head inside tile block 0 of the slot's range
+    int32_t q_row;          // first row of the item's query group in q / out  (request row + q_tok0)
+    int32_t partial_idx;    // -1: writes the final output; else slot in the partial workspace
+    int32_t tile_begin, tile_end;
+    int32_t kv_end;         // keys visible to the group's last query token
+    int16_t head0;          // first query head of the group (kv_head * G + g0)
+    uint8_t n_q_tok, n_g;   // rows = n_q_tok * n_g <= kMaxRows
 };
+static_assert(sizeof(DevItem) == 32, "DevItem layout");
 
 struct CombineDesc {        // one per split unit
     int32_t partial_begin, n_parts;
@@ -47,7 +52,7 @@ struct CombineDesc {        // one per split unit
     int32_t n_q_tok, n_g;
 };
 
-struct AppendDesc {         // one per request of an append / gather call
+struct AppendDesc {         // one per request of an append call
     uint64_t base;
     int32_t pos0;           // first token position written
     int32_t row0;           // first source row
@@ -56,18 +61,18 @@ struct AppendDesc {         // one per request of an append / gather call
 };
 
 struct AttnLaunch {
-    const xllm_work_item *items;  // device
-    const int32_t *cta_begin;     // device [n_ctas + 1]
-    const ReqDesc *reqs;          // device
+    const DevItem *items;         // device, grouped by CTA
     const void *q;
     void *out;
     float *lse_out;               // may be null
     float *part_o;                // [n_partials][kMaxRows][D] fp32
     float *part_lse;              // [n_partials][kMaxRows]    (log2 domain)
-    int32_t *error_flag;          // device; set non-zero when a bounded wait expires
+    int32_t *error_flag;          // host-mapped; set non-zero when a bounded wait expires
+    unsigned long long *trace;    // optional per-CTA cycle counters (debug), may be null
     int32_t n_q_heads, n_kv_heads, head_dim;
     float scale_log2;             // scale * log2(e)
     int32_t n_ctas;
+    int32_t cta_begin[kMaxCtas + 1];  // CTA c owns items [cta_begin[c], cta_begin[c+1])
 };
 
 struct CombineLaunch {
@@ -80,12 +85,14 @@ struct CombineLaunch {
     int32_t n_q_heads, head_dim;
 };
 
+constexpr int32_t kTraceWords = 16;  // per-CTA words of the optional trace buffer
+
 // kernels.cu
 int attention_smem_bytes(int32_t head_dim);
 int configure_kernels(int32_t head_dim);  // cudaFuncSetAttribute for the dynamic shared memory; returns cudaError
 int launch_attention(const AttnLaunch &p, void *stream);
 int launch_combine(const CombineLaunch &p, void *stream);
-int launch_append(const AppendDesc *descs, int32_t n_req, int32_t n_rows, const void *k_new, const void *v_new,
+int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *k_new, const void *v_new,
                   int32_t n_kv_heads, int32_t head_dim, void *stream);
 int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,
                   int32_t head_dim, void *stream);

@@ -1,18 +1,20 @@
 // CUDA kernels of libxllm_attn.so (sm_100a): KV append / gather, split-KV attention, LSE combine.
 //
 // Attention kernel in one paragraph.  One persistent CTA per SM walks its run of work items (see
-// partition.cpp).  Warp 8 is the producer: an elected lane streams head tiles (K then V of one KV head
-// for 64 tokens, one contiguous run of the slot's range) into a ring of shared-memory stages with
-// cp.async.bulk + mbarrier transaction counts, and the query rows of the next item into a double
-// buffer, never draining the ring between items.  Warps 0-7 are consumers in two groups of four that
-// take alternate tiles; inside a group each warp owns 16 tokens of the tile and keeps its own online
-// softmax state (running max, sum, fp32 output accumulator) for all query rows of the GQA group
-// (rows = heads of the group x query tokens <= 16), so every K/V byte is fetched from HBM once for
-// all of them.  Q.K^T and P.V run on mma.sync m16n8k16 bf16 (the work is HBM bound: ~rows flop/byte).
-// At the end of an item each consumer warp drops its state into shared memory and moves on; warps 9-11
-// (epilogue) merge the eight states and write either the final bf16 output or an fp32 partial (+ log2-domain
-// LSE) while the consumers already work on the next item.  The speculative-verification
-// causal mask only touches the tiles that hold the newest q_len tokens.
+// partition.cpp).  Warp 8 is the producer: an elected lane streams head tiles (K half, then V half, of one
+// KV head for 64 tokens; each half is one contiguous run of the slot's range) into a ring of shared-memory
+// half stages with cp.async.bulk + mbarrier transaction counts, and the query rows of the next item into
+// a double buffer, never draining the ring between items.  Warps 0-7 are consumers in two groups of four
+// that take alternate tiles.  Inside a group, warp w computes the scores of tokens 16w..16w+15 of the tile
+// for all query rows of the GQA group (rows = heads of the group x query tokens <= 16), the four warps agree
+// on the tile's row maxima through shared memory, exchange their bf16 softmax weights, and then each warp
+// accumulates P.V for ALL 64 tokens into its own quarter of the head dimension.  A group therefore keeps
+// one online-softmax state (running max, sum, fp32 output) spread over its warps, and every K/V byte is
+// fetched from HBM once for all query rows.  Q.K^T and P.V run on mma.sync m16n8k16 bf16 (the work is HBM
+// bound: ~rows flop/byte).  At the end of an item the two group states go to shared memory and warps 9-11
+// (epilogue) merge them and write either the final bf16 output or an fp32 partial (+ log2-domain LSE) while
+// the consumers already work on the next item.  The speculative-verification causal mask only touches the
+// tiles that hold the newest q_len tokens.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -37,22 +39,36 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // a bounded wait gi
 template <int D>
 struct Cfg {
     static constexpr int kPanels = D / 64;
-    static constexpr int kHeadTile = 2 * kPanels * kPanelBytes;      // K + V of one head, 64 tokens
     static constexpr int kHalfTile = kPanels * kPanelBytes;          // K or V of one head, 64 tokens
-    static constexpr int kStages = 4 * (128 / D);                    // tiles of ring capacity
-    static constexpr int kHalfStages = 2 * kStages;                  // K and V halves are acquired and released separately
+    // Ring slots, acquired and released per half tile.  Each consumer group owns a ring of its own, so the uses of
+    // a slot are always consumed by the same four warps in order: a waiter then never sees an mbarrier more than
+    // one phase away from the one it wants, which the one-bit phase parity of mbarrier.try_wait requires.
+    static constexpr int kSlotsA = 6 * (128 / D);                    // group 0 (even tiles)
+    static constexpr int kSlotsB = 5 * (128 / D);                    // group 1 (odd tiles)
+    static constexpr int kHalfStages = kSlotsA + kSlotsB;
+    // slot and phase of half `x` (0 = K, 1 = V) of the j-th tile of group g
+    __device__ static __forceinline__ void slot_of(uint32_t g, uint32_t j, uint32_t x, uint32_t &slot, uint32_t &phase) {
+        const uint32_t hl = 2 * j + x, n = g ? kSlotsB : kSlotsA;
+        slot = (g ? kSlotsA : 0) + hl % n;
+        phase = (hl / n) & 1;
+    }
     static constexpr int kQPitch = D * 2 + 16;                       // bytes, padded against bank conflicts
     static constexpr int kOPitch = D + 8;                            // floats
+    static constexpr int kPPitch = T * 2 + 16;                       // bytes per row of the bf16 weight tile
+    static constexpr int kColsPerWarp = D / 4;                       // head-dim columns a warp accumulates
     static constexpr int kOffStages = 0;
-    static constexpr int kOffMergeO = kOffStages + kStages * kHeadTile;
-    static constexpr int kOffMergeM = kOffMergeO + kConsumerWarps * kMaxRows * kOPitch * 4;
-    static constexpr int kOffMergeL = kOffMergeM + kConsumerWarps * kMaxRows * 4;
-    static constexpr int kOffQ = kOffMergeL + kConsumerWarps * kMaxRows * 4;
+    static constexpr int kOffMergeO = kOffStages + kHalfStages * kHalfTile;      // [2 groups][16 rows][kOPitch] fp32
+    static constexpr int kOffMergeM = kOffMergeO + 2 * kMaxRows * kOPitch * 4;   // [2][16]
+    static constexpr int kOffMergeL = kOffMergeM + 2 * kMaxRows * 4;             // [2][4 warps][16]
+    static constexpr int kOffMax = kOffMergeL + 2 * 4 * kMaxRows * 4;            // [2 groups][2 bufs][4 warps][16] tile row maxima
+    static constexpr int kOffP = kOffMax + 2 * 2 * 4 * kMaxRows * 4;             // [2 groups][2 bufs][16 rows][kPPitch]
+    static constexpr int kOffQ = kOffP + 2 * 2 * kMaxRows * kPPitch;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
     static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(DevItem);
     static constexpr int kNumBars = 2 * kHalfStages + 6;
     static constexpr int kOffFlags = kOffBars + kNumBars * 8;
     static constexpr int kSmemBytes = kOffFlags + 16;
+    static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
 
 // ---- PTX wrappers --------------------------------------------------------------------------------------
@@ -129,18 +145,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// ---- one 16-token slice of a tile, all query rows ---------------------------------------------------------
-// Phase 1 (needs the K half of the tile): scores, mask, online-softmax update; returns the bf16 weights as an MMA
-// A fragment.  HALF: the item has at most 8 rows, so rows 8..15 of the MMA tile are padding and are skipped.
+__device__ __forceinline__ void group_bar(int group) {
+    __syncwarp();  // the barrier instruction is warp-aligned: make sure the lanes have re-converged
+    asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
+}
+
+// ---- split-KV attention ---------------------------------------------------------------------------------
+// Warp roles: 0-7 consumers (two groups of four taking alternate tiles), 8 producer (bulk copies), 9-11 epilogue
+// (merge the two group states of a finished item and write its result while the consumers go on).
+// MASK: the tile holds tokens some row must not see, or tokens past the end (stale bytes).  HALF: the item has at
+// most 8 rows, so rows 8..15 of the MMA tile are padding and their softmax is skipped.
 template <int D, bool MASK, bool HALF>
-__device__ __forceinline__ void slice_scores(uint32_t kstage, int wslice, int lane, const uint32_t (&qf)[D / 16][4],
-                                             float (&o)[D / 8][4], float (&m)[2], float (&l)[2], float scale_log2,
-                                             int tok_base, int limit_lo, int limit_hi, uint32_t (&pa)[4]) {
-    const int swz = lane & 7;
-    // two accumulation chains per 8-token block (even / odd k-steps) to shorten the dependent MMA chain
+__device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, uint32_t bar_k_full, uint32_t bar_v_full,
+                                             uint32_t bar_k_empty, uint32_t bar_v_empty, uint32_t ph_k, uint32_t ph_v, int group, int wslice,
+                                             int lane, const uint32_t (&qf)[D / 16][4], float (&o)[D / 32][4], float (&m)[2],
+                                             float (&l)[2], float scale_log2, int tile_tok0, int limit_lo, int limit_hi,
+                                             int kv_end, float *mxs, uint32_t ps, bool &live, volatile int *abort_flag,
+                                             int32_t *error_flag) {
+    const int swz = lane & 7, q4 = lane & 3, g8 = lane >> 2;
+    const int tok_base = tile_tok0 + wslice * 16;
+    const bool work = tok_base < kv_end;  // the slice holds at least one fetched token
+    live = mbar_wait(bar_k_full, ph_k, abort_flag, error_flag, 4) && live;
+
+    // ---- scores of this warp's 16 tokens; two accumulation chains per 8-token block ----
     float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    float s2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    {
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+    if (live && work) {
+        float s2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
         const int r = wslice * 16 + (lane & 7) + ((lane >> 4) << 3);
         const int csel = (lane >> 3) & 1;
         const uint32_t row_addr = kstage + r * 128;
@@ -159,47 +190,70 @@ __device__ __forceinline__ void slice_scores(uint32_t kstage, int wslice, int la
         for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) s[nt][e] += s2[nt][e];
-    }
-    const int q4 = lane & 3;
-    if (MASK) {
+        if (MASK) {
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
+            for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int e = 0; e < (HALF ? 2 : 4); ++e) {
-                const int tok = tok_base + nt * 8 + 2 * q4 + (e & 1);
-                if (tok >= ((e < 2) ? limit_lo : limit_hi)) s[nt][e] = -INFINITY;
-            }
+                for (int e = 0; e < (HALF ? 2 : 4); ++e) {
+                    const int tok = tok_base + nt * 8 + 2 * q4 + (e & 1);
+                    if (tok >= ((e < 2) ? limit_lo : limit_hi)) s[nt][e] = -INFINITY;
+                }
+        }
+        mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        if (!HALF) {
+            mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        }
     }
-    float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_k_empty);  // this warp is done with the K half
+    if (q4 == 0) {
+        mxs[wslice * kMaxRows + g8] = mx0;
+        if (!HALF) mxs[wslice * kMaxRows + g8 + 8] = mx1;
+    }
+    group_bar(group);  // (1) the four slices' row maxima are visible
+
+    // ---- shared running max, weights of this slice, exchange of the bf16 weight tile ----
+    mx0 = fmaxf(fmaxf(mxs[g8], mxs[kMaxRows + g8]), fmaxf(mxs[2 * kMaxRows + g8], mxs[3 * kMaxRows + g8]));
     const float mn0 = fmaxf(m[0], mx0 * scale_log2);
     const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0;
     const float a0 = exp2f(m[0] - ms0);
     m[0] = mn0;
     float ms1 = 0.f, a1 = 1.f;
     if (!HALF) {
-        float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        mx1 = fmaxf(fmaxf(mxs[g8 + 8], mxs[kMaxRows + g8 + 8]), fmaxf(mxs[2 * kMaxRows + g8 + 8], mxs[3 * kMaxRows + g8 + 8]));
         const float mn1 = fmaxf(m[1], mx1 * scale_log2);
         ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
         a1 = exp2f(m[1] - ms1);
         m[1] = mn1;
     }
-    float p[2][4];
+    l[0] *= a0;
+    if (!HALF) l[1] *= a1;
+    if (live && work) {
+        float p[2][4];
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-        p[nt][0] = exp2f(fmaf(s[nt][0], scale_log2, -ms0));
-        p[nt][1] = exp2f(fmaf(s[nt][1], scale_log2, -ms0));
-        p[nt][2] = HALF ? 0.f : exp2f(fmaf(s[nt][2], scale_log2, -ms1));
-        p[nt][3] = HALF ? 0.f : exp2f(fmaf(s[nt][3], scale_log2, -ms1));
+        for (int nt = 0; nt < 2; ++nt) {
+            p[nt][0] = exp2f(fmaf(s[nt][0], scale_log2, -ms0));
+            p[nt][1] = exp2f(fmaf(s[nt][1], scale_log2, -ms0));
+            p[nt][2] = HALF ? 0.f : exp2f(fmaf(s[nt][2], scale_log2, -ms1));
+            p[nt][3] = HALF ? 0.f : exp2f(fmaf(s[nt][3], scale_log2, -ms1));
+        }
+        l[0] += (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
+        if (!HALF) l[1] += (p[0][2] + p[0][3]) + (p[1][2] + p[1][3]);
+        const uint32_t dst = ps + g8 * Cfg<D>::kPPitch + (wslice * 16 + 2 * q4) * 2;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + nt * 16), "r"(pack_bf16(p[nt][0], p[nt][1])) : "memory");
+            if (!HALF)
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + 8 * Cfg<D>::kPPitch + nt * 16), "r"(pack_bf16(p[nt][2], p[nt][3])) : "memory");
+        }
     }
-    l[0] = l[0] * a0 + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
-    if (!HALF) l[1] = l[1] * a1 + (p[0][2] + p[0][3] + p[1][2] + p[1][3]);
     if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {  // the running maximum moved: rescale the accumulator
 #pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt) {
+        for (int nt = 0; nt < D / 32; ++nt) {
             o[nt][0] *= a0;
             o[nt][1] *= a0;
             if (!HALF) {
@@ -208,45 +262,48 @@ __device__ __forceinline__ void slice_scores(uint32_t kstage, int wslice, int la
             }
         }
     }
-    pa[0] = pack_bf16(p[0][0], p[0][1]);
-    pa[1] = HALF ? 0u : pack_bf16(p[0][2], p[0][3]);
-    pa[2] = pack_bf16(p[1][0], p[1][1]);
-    pa[3] = HALF ? 0u : pack_bf16(p[1][2], p[1][3]);
-}
+    group_bar(group);  // (2) the weight tile is complete
+    live = mbar_wait(bar_v_full, ph_v, abort_flag, error_flag, 7) && live;
 
-// Phase 2 (needs the V half): O += P . V for the slice's 16 tokens.
-template <int D, bool MASK>
-__device__ __forceinline__ void slice_pv(uint32_t vstage, int wslice, int lane, const uint32_t (&pa)[4], float (&o)[D / 8][4],
-                                         int tok_base, int kv_end) {
-    const int swz = lane & 7, q4 = lane & 3;
-    uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
-    if (MASK) {  // V rows never written by append may hold anything: force them to zero (0 * NaN would poison O)
-        const int t0 = tok_base + 2 * q4;
-        vmask0 = (t0 < kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < kv_end ? 0xffff0000u : 0u);
-        vmask1 = (t0 + 8 < kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < kv_end ? 0xffff0000u : 0u);
-    }
-    const int r = wslice * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-    const int csel = lane >> 4;
-    const uint32_t row_addr = vstage + r * 128;
+    // ---- O[:, this warp's columns] += P[16 x 64] . V[64 x columns] ----
+    if (live) {
+        const int n_ks = MASK ? min(4, (kv_end - tile_tok0 + 15) >> 4) : 4;  // 16-token steps that hold fetched tokens
+        const uint32_t p_addr = ps + ((lane & 7) + (((lane >> 3) & 1) << 3)) * Cfg<D>::kPPitch + ((lane >> 4) << 4);
+        const int vr = (lane & 7) + (((lane >> 3) & 1) << 3);
+        const int csel = lane >> 4;
 #pragma unroll
-    for (int n2 = 0; n2 < D / 16; ++n2) {
-        const int cg = 2 * n2 + csel;
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
-        if (MASK) {
-            b0 &= vmask0;
-            b1 &= vmask1;
-            b2 &= vmask0;
-            b3 &= vmask1;
+        for (int kk = 0; kk < 4; ++kk) {
+            if (MASK && kk >= n_ks) break;
+            uint32_t pa[4];
+            ldsm_x4(pa[0], pa[1], pa[2], pa[3], p_addr + kk * 32);
+            if (HALF) pa[1] = pa[3] = 0u;
+            uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
+            if (MASK) {  // V rows never written by append may hold anything: force them to zero (0 * NaN would poison O)
+                const int t0 = tile_tok0 + kk * 16 + 2 * q4;
+                vmask0 = (t0 < kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < kv_end ? 0xffff0000u : 0u);
+                vmask1 = (t0 + 8 < kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < kv_end ? 0xffff0000u : 0u);
+            }
+            const uint32_t row_addr = vstage + (kk * 16 + vr) * 128;
+#pragma unroll
+            for (int n2 = 0; n2 < D / 64; ++n2) {
+                const int cg = wslice * (D / 32) + 2 * n2 + csel;  // 8-column chunk of the head dimension
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
+                if (MASK) {
+                    b0 &= vmask0;
+                    b1 &= vmask1;
+                    b2 &= vmask0;
+                    b3 &= vmask1;
+                }
+                mma_bf16(o[2 * n2], pa, b0, b1);
+                mma_bf16(o[2 * n2 + 1], pa, b2, b3);
+            }
         }
-        mma_bf16(o[2 * n2], pa, b0, b1);
-        mma_bf16(o[2 * n2 + 1], pa, b2, b3);
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_v_empty);  // this warp is done with the V half
 }
 
-// ---- split-KV attention ---------------------------------------------------------------------------------
-// Warp roles: 0-7 consumers (two groups of four taking alternate tiles), 8 producer (bulk copies), 9-11 epilogue
-// (merge the eight per-warp states of a finished item and write its result while the consumers go on).
 template <int D, bool TRACE>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnLaunch p) {
     using C = Cfg<D>;
@@ -259,7 +316,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const uint32_t bar_empty = bar_full + C::kHalfStages * 8;         // [kHalfStages] ... consumed (4 warps)
     const uint32_t bar_qfull = bar_empty + C::kHalfStages * 8;        // [2] query rows landed
     const uint32_t bar_qempty = bar_qfull + 16;                       // [2] query rows loaded to registers (8 warps)
-    const uint32_t bar_mfull = bar_qempty + 16;                       // per-warp states of an item written (8 warps)
+    const uint32_t bar_mfull = bar_qempty + 16;                       // group states of an item written (8 warps)
     const uint32_t bar_mempty = bar_mfull + 8;                        // ... and read by the epilogue (3 warps)
     const unsigned long long t_start = TRACE ? clock64() : 0ull;
     const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
@@ -280,11 +337,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
-    const int64_t tile_block = (int64_t)p.n_kv_heads * C::kHeadTile;
+    const int64_t tile_block = (int64_t)p.n_kv_heads * 2 * C::kHalfTile;
     uint32_t fill = 0;      // tiles issued / consumed so far by this CTA (same sequence in every warp)
     uint32_t item_seq = 0;  // items started so far
-    unsigned long long tr_wait_full = 0, tr_compute = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0,
-                       tr_epi = 0;
+    unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0;
 
     for (int batch_lo = item_lo; batch_lo < item_hi; batch_lo += kItemBatch) {
         const int nb = min(kItemBatch, item_hi - batch_lo);
@@ -311,13 +367,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     }
                     const char *kv = reinterpret_cast<const char *>(it.kv);
                     for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
-                        const uint32_t s = fill % C::kStages, ph = (fill / C::kStages) & 1;
                         const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);
                         const uint32_t bytes = rows * 128;
                         const char *src = kv + (int64_t)tile * tile_block;
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {  // K half, then V half
-                            const uint32_t hs = 2 * s + half;
+                            uint32_t hs, ph;
+                            C::slot_of(fill & 1, fill >> 1, half, hs, ph);
                             const unsigned long long t0 = TRACE ? clock64() : 0ull;
                             if (!mbar_wait(bar_empty + hs * 8, ph ^ 1, abort_flag, p.error_flag, 2)) continue;
                             if (TRACE) tr_wait_empty += clock64() - t0;
@@ -337,9 +393,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             // ================= consumers =================
             const int group = warp >> 2, wslice = warp & 3;
             const int g8 = lane >> 2, q4 = lane & 3;
-            float *merge_o = reinterpret_cast<float *>(smem + C::kOffMergeO);
-            float *merge_m = reinterpret_cast<float *>(smem + C::kOffMergeM);
-            float *merge_l = reinterpret_cast<float *>(smem + C::kOffMergeL);
+            float *merge_o = reinterpret_cast<float *>(smem + C::kOffMergeO) + group * kMaxRows * C::kOPitch;
+            float *merge_m = reinterpret_cast<float *>(smem + C::kOffMergeM) + group * kMaxRows;
+            float *merge_l = reinterpret_cast<float *>(smem + C::kOffMergeL) + (group * 4 + wslice) * kMaxRows;
+            float *mx_base = reinterpret_cast<float *>(smem + C::kOffMax) + group * (2 * 4 * kMaxRows);
+            const uint32_t p_base = smem_base + C::kOffP + group * (2 * kMaxRows * C::kPPitch);
+            uint32_t my_tiles = 0;  // tiles this group has processed: selects the double buffer of maxima / weights
             for (int i = 0; i < nb; ++i) {
                 const DevItem it = sitems[i];
                 const int n_rows = it.n_q_tok * it.n_g;
@@ -365,83 +424,64 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 const int limit_lo = (g8 < n_rows) ? row_limit0 + g8 / it.n_g : 0;
                 const int limit_hi = (g8 + 8 < n_rows) ? row_limit0 + (g8 + 8) / it.n_g : 0;
                 const bool half = n_rows <= 8;
-                float o[D / 8][4];
+                float o[D / 32][4];
 #pragma unroll
-                for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+                for (int nt = 0; nt < D / 32; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
                 float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
 
+                t0 = TRACE ? clock64() : 0ull;
                 for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
                     if ((int)(fill & 1) != group) continue;
-                    const uint32_t s = fill % C::kStages, ph = (fill / C::kStages) & 1;
-                    const uint32_t bk = bar_full + (2 * s) * 8, bv = bk + 8;
-                    const uint32_t kstage = smem_base + C::kOffStages + (2 * s) * C::kHalfTile, vstage = kstage + C::kHalfTile;
-                    const int tok_base = tile * T + wslice * 16;
-                    const bool work = tok_base < it.kv_end;
+                    uint32_t sk, sv, phk, phv;
+                    C::slot_of(group, fill >> 1, 0, sk, phk);
+                    C::slot_of(group, fill >> 1, 1, sv, phv);
+                    const uint32_t kstage = smem_base + C::kOffStages + sk * C::kHalfTile;
+                    const uint32_t vstage = smem_base + C::kOffStages + sv * C::kHalfTile;
+                    float *mxs = mx_base + (my_tiles & 1) * (4 * kMaxRows);
+                    const uint32_t ps = p_base + (my_tiles & 1) * (kMaxRows * C::kPPitch);
+                    ++my_tiles;
                     const bool mask = tile * T + T > row_limit0;
-                    uint32_t pa[4];
-                    t0 = TRACE ? clock64() : 0ull;
-                    live = mbar_wait(bk, ph, abort_flag, p.error_flag, 4) && live;
-                    if (TRACE) {
-                        const unsigned long long t1 = clock64();
-                        tr_wait_full += t1 - t0;
-                        if (!tr_first) tr_first = t1 - t_start;
-                        t0 = t1;
+#define XLLM_TILE(MASK_, HALF_)                                                                                              \
+    consume_tile<D, MASK_, HALF_>(kstage, vstage, bar_full + sk * 8, bar_full + sv * 8, bar_empty + sk * 8, bar_empty + sv * 8, \
+                                  phk, phv, group, wslice, lane, qf, o, m, l, p.scale_log2, tile * T, limit_lo, limit_hi, it.kv_end, \
+                                  mxs, ps, live, abort_flag, p.error_flag)
+                    if (half) {
+                        if (mask) XLLM_TILE(true, true); else XLLM_TILE(false, true);
+                    } else {
+                        if (mask) XLLM_TILE(true, false); else XLLM_TILE(false, false);
                     }
-                    if (live && work) {
-                        if (half) {
-                            if (mask) slice_scores<D, true, true>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
-                            else slice_scores<D, false, true>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
-                        } else {
-                            if (mask) slice_scores<D, true, false>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
-                            else slice_scores<D, false, false>(kstage, wslice, lane, qf, o, m, l, p.scale_log2, tok_base, limit_lo, limit_hi, pa);
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty + (2 * s) * 8);      // K half is free again
-                    if (TRACE) {
-                        const unsigned long long t1 = clock64();
-                        tr_compute += t1 - t0;
-                        t0 = t1;
-                    }
-                    live = mbar_wait(bv, ph, abort_flag, p.error_flag, 7) && live;
-                    if (TRACE) {
-                        const unsigned long long t1 = clock64();
-                        tr_wait_full += t1 - t0;
-                        t0 = t1;
-                    }
-                    if (live && work) {
-                        if (mask) slice_pv<D, true>(vstage, wslice, lane, pa, o, tok_base, it.kv_end);
-                        else slice_pv<D, false>(vstage, wslice, lane, pa, o, tok_base, it.kv_end);
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty + (2 * s + 1) * 8);  // V half is free again
-                    if (TRACE) tr_compute += clock64() - t0;
+#undef XLLM_TILE
+                    if (TRACE && !tr_first) tr_first = clock64() - t_start;
+                }
+                if (TRACE) {
+                    const unsigned long long t1 = clock64();
+                    tr_tiles += t1 - t0;
+                    t0 = t1;
                 }
 
-                // ---- hand the warp's state to the epilogue warps and go on with the next item ----
-                t0 = TRACE ? clock64() : 0ull;
+                // ---- hand the group's state to the epilogue warps and go on with the next item ----
                 l[0] += __shfl_xor_sync(0xffffffffu, l[0], 1);
                 l[1] += __shfl_xor_sync(0xffffffffu, l[1], 1);
                 l[0] += __shfl_xor_sync(0xffffffffu, l[0], 2);
                 l[1] += __shfl_xor_sync(0xffffffffu, l[1], 2);
                 mbar_wait(bar_mempty, (seq + 1) & 1, abort_flag, p.error_flag, 5);  // previous item's states were read
                 if (q4 == 0) {
-                    merge_m[warp * kMaxRows + g8] = m[0];
-                    merge_l[warp * kMaxRows + g8] = l[0];
+                    merge_l[g8] = l[0];
+                    if (wslice == 0) merge_m[g8] = m[0];
                     if (!half) {
-                        merge_m[warp * kMaxRows + g8 + 8] = m[1];
-                        merge_l[warp * kMaxRows + g8 + 8] = l[1];
+                        merge_l[g8 + 8] = l[1];
+                        if (wslice == 0) merge_m[g8 + 8] = m[1];
                     }
                 }
                 {
-                    // always written: a warp that saw no visible key holds exact zeros, which the epilogue weighs by 0
-                    float *dst = merge_o + (warp * kMaxRows + g8) * C::kOPitch + 2 * q4;
+                    // always written: a group that saw no visible key holds exact zeros, which the epilogue weighs by 0
+                    float *dst = merge_o + g8 * C::kOPitch + wslice * C::kColsPerWarp + 2 * q4;
 #pragma unroll
-                    for (int nt = 0; nt < D / 8; ++nt)
+                    for (int nt = 0; nt < D / 32; ++nt)
                         *reinterpret_cast<float2 *>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
                     if (!half) {
 #pragma unroll
-                        for (int nt = 0; nt < D / 8; ++nt)
+                        for (int nt = 0; nt < D / 32; ++nt)
                             *reinterpret_cast<float2 *>(dst + 8 * C::kOPitch + nt * 8) = make_float2(o[nt][2], o[nt][3]);
                     }
                 }
@@ -464,39 +504,29 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 const unsigned long long t0 = TRACE ? clock64() : 0ull;
                 for (int idx = et; live && idx < n_rows * kC4; idx += kEpilogueThreads) {
                     const int row = idx / kC4, c4 = idx - row * kC4;
-                    float mw[kConsumerWarps];
-                    float M = -INFINITY;
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w) {
-                        mw[w] = merge_m[w * kMaxRows + row];
-                        M = fmaxf(M, mw[w]);
-                    }
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    float L = 0.f;
-                    {
-                        const float Ms = (M == -INFINITY) ? 0.f : M;
-#pragma unroll
-                        for (int w = 0; w < kConsumerWarps; ++w) {
-                            const float wgt = exp2f(mw[w] - Ms);  // 0 for a warp that saw no visible key (its O row is all zeros)
-                            L += wgt * merge_l[w * kMaxRows + row];
-                            const float4 v = *reinterpret_cast<const float4 *>(merge_o + (w * kMaxRows + row) * C::kOPitch + c4 * 4);
-                            acc.x += wgt * v.x;
-                            acc.y += wgt * v.y;
-                            acc.z += wgt * v.z;
-                            acc.w += wgt * v.w;
-                        }
-                    }
+                    const float mA = merge_m[row], mB = merge_m[kMaxRows + row];
+                    const float lA = (merge_l[row] + merge_l[kMaxRows + row]) + (merge_l[2 * kMaxRows + row] + merge_l[3 * kMaxRows + row]);
+                    const float lB = (merge_l[4 * kMaxRows + row] + merge_l[5 * kMaxRows + row]) +
+                                     (merge_l[6 * kMaxRows + row] + merge_l[7 * kMaxRows + row]);
+                    const float4 oA = *reinterpret_cast<const float4 *>(merge_o + row * C::kOPitch + c4 * 4);
+                    const float4 oB = *reinterpret_cast<const float4 *>(merge_o + (kMaxRows + row) * C::kOPitch + c4 * 4);
+                    const float M = fmaxf(mA, mB);
+                    const float Ms = (M == -INFINITY) ? 0.f : M;
+                    const float wA = exp2f(mA - Ms), wB = exp2f(mB - Ms);  // 0 for a group that saw no visible key
+                    const float L = wA * lA + wB * lB;
                     const float inv = (L > 0.f) ? 1.f / L : 0.f;
                     const float lse2 = (L > 0.f) ? M + log2f(L) : -INFINITY;
+                    const float4 acc = make_float4((wA * oA.x + wB * oB.x) * inv, (wA * oA.y + wB * oB.y) * inv,
+                                                   (wA * oA.z + wB * oB.z) * inv, (wA * oA.w + wB * oB.w) * inv);
                     if (it.partial_idx >= 0) {
                         float *dst = p.part_o + ((int64_t)it.partial_idx * kMaxRows + row) * D + c4 * 4;
-                        *reinterpret_cast<float4 *>(dst) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                        *reinterpret_cast<float4 *>(dst) = acc;
                         if (c4 == 0) p.part_lse[(int64_t)it.partial_idx * kMaxRows + row] = lse2;
                     } else {
                         const int ti = row / it.n_g, gi = row - ti * it.n_g;
                         const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
                         *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
-                            make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                            make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
                         if (c4 == 0 && p.lse_out) p.lse_out[off] = lse2 * 0.69314718055994531f;
                     }
                 }
@@ -509,15 +539,19 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         item_seq += nb;
     }
 
+    // trace layout (16 words per CTA): 0 cycles of warp 0, 1 cycles to its first finished tile, 2 cycles in tile loops
+    // (warp 0), 3 unused, 4 waiting for query rows, 5 item hand-off incl. waiting for the epilogue, 6 items, 7 tiles,
+    // 8/10 the same as 2/5 for warp 4, 11 producer cycles waiting for free ring slots, 12 producer cycles,
+    // 13 epilogue busy cycles, 14 epilogue cycles, 15 nanoseconds of warp 0 (global timer).
     if (TRACE && lane == 0 && (warp == 0 || warp == 4 || warp == kProducerWarp || warp == kEpilogueWarp0)) {
         unsigned long long *tr = p.trace + (int64_t)blockIdx.x * kTraceWords;
         const unsigned long long total = clock64() - t_start;
         if (warp == 0) {
-            tr[0] = total; tr[1] = tr_first; tr[2] = tr_wait_full; tr[3] = tr_compute; tr[4] = tr_wait_q; tr[5] = tr_switch;
+            tr[0] = total; tr[1] = tr_first; tr[2] = tr_tiles; tr[3] = 0; tr[4] = tr_wait_q; tr[5] = tr_switch;
             tr[6] = (unsigned long long)(item_hi - item_lo); tr[7] = fill;
             tr[15] = globaltimer_ns() - g_start;
         } else if (warp == 4) {
-            tr[8] = tr_wait_full; tr[9] = tr_compute; tr[10] = tr_switch;
+            tr[8] = tr_tiles; tr[9] = 0; tr[10] = tr_switch;
         } else if (warp == kProducerWarp) {
             tr[11] = tr_wait_empty; tr[12] = total;
         } else {
@@ -530,11 +564,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     __syncthreads();
     if (*abort_flag && warp == kProducerWarp && lane == 0) {
         const unsigned long long t0 = globaltimer_ns();
-        for (uint32_t back = 0; back < (uint32_t)C::kStages && back < fill; ++back) {
-            const uint32_t f = fill - 1 - back, s = f % C::kStages, ph = (f / C::kStages) & 1;
-            for (uint32_t hs = 2 * s; hs < 2 * s + 2; ++hs)
+        for (uint32_t g = 0; g < 2; ++g) {
+            const uint32_t tiles_g = (fill + 1 - g) / 2, halves_g = 2 * tiles_g, n = g ? C::kSlotsB : C::kSlotsA;
+            for (uint32_t back = 0; back < n && back < halves_g; ++back) {
+                const uint32_t hl = halves_g - 1 - back;
+                uint32_t hs, ph;
+                C::slot_of(g, hl >> 1, hl & 1, hs, ph);
                 while (!mbar_try_wait(bar_full + hs * 8, ph) && globaltimer_ns() - t0 < kWaitLimitNs) {
                 }
+            }
         }
     }
 }

@@ -211,16 +211,18 @@ class Replica:
         torch.cuda.synchronize()
         self.pre = (self.kv - self.ql).astype(np.int64)
         self.decode_only = bool((self.ql == 1).all())
+        self.stream = torch.cuda.current_stream().cuda_stream
 
     def step(self, i: int, q=None, k_new=None, v_new=None):
         ctx, slots = self.ctx, self.slots[i % self.copies]
         q = self.q if q is None else q
         ctx.kv_map_pages_many(slots, self.kv)                              # a1: pages for the tokens about to be written
-        ctx.kv_append(slots, self.ql, self.k_new if k_new is None else k_new, self.v_new if v_new is None else v_new)  # a2
+        ctx.kv_append(slots, self.ql, self.k_new if k_new is None else k_new, self.v_new if v_new is None else v_new,
+                      self.stream)                                         # a2
         if self.decode_only:                                               # a3 + a4 + a5
-            ctx.decode_attention(slots, q, self.out, None, self.s.scale)
+            ctx.decode_attention(slots, q, self.out, None, self.s.scale, self.stream)
         else:
-            ctx.verify_attention(slots, self.ql, q, self.out, None, self.s.scale)
+            ctx.verify_attention(slots, self.ql, q, self.out, None, self.s.scale, self.stream)
         ctx.kv_set_len_many(slots, self.pre)                               # back to the named context lengths
 
     def step_e2e(self, i: int):

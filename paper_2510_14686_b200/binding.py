@@ -80,8 +80,8 @@ EXPORTS = {
     "xllm_sync_check": (ctypes.c_int32, [_ctxp, _vp]),
     "xllm_kv_reserve": (ctypes.c_int32, [_ctxp, ctypes.c_int64, ctypes.c_int64, _i32p]),
     "xllm_kv_map_pages": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
-    "xllm_kv_map_pages_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i64p]),
-    "xllm_kv_set_len_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i64p]),
+    "xllm_kv_map_pages_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp]),
+    "xllm_kv_set_len_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp]),
     "xllm_kv_release": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int32]),
     "xllm_kv_set_len": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
     "xllm_kv_slot_info": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.POINTER(SlotInfo)]),
@@ -89,10 +89,10 @@ EXPORTS = {
     "xllm_debug_read_slot": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
     "xllm_debug_read_page": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
     "xllm_debug_read_trace": (ctypes.c_int32, [_ctxp, ctypes.POINTER(ctypes.c_uint64), ctypes.c_int32, _i32p]),
-    "xllm_kv_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i32p, _vp, _vp, _vp]),
+    "xllm_kv_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp]),
     "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
-    "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _vp, _vp, _vp, ctypes.c_float, _vp]),
-    "xllm_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _i32p, _i32p, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.POINTER(WorkItem), ctypes.c_int32, _i32p, _i32p, _i32p, _i32p]),
     "xllm_get_stats": (ctypes.c_int32, [_ctxp, ctypes.POINTER(Stats)]),
@@ -104,7 +104,15 @@ for _name, (_res, _args) in EXPORTS.items():
 
 
 def _i32(a) -> np.ndarray:
+    if isinstance(a, np.ndarray) and a.dtype == np.int32 and a.flags.c_contiguous:
+        return a
     return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i64(a) -> np.ndarray:
+    if isinstance(a, np.ndarray) and a.dtype == np.int64 and a.flags.c_contiguous:
+        return a
+    return np.ascontiguousarray(a, dtype=np.int64)
 
 
 def _ptr(t) -> int:
@@ -192,12 +200,12 @@ class Context:
         self._check(_lib.xllm_kv_map_pages(self._ctx, slot, min_tokens))
 
     def kv_map_pages_many(self, slots, min_tokens):
-        s, t = _i32(slots), np.ascontiguousarray(min_tokens, dtype=np.int64)
-        self._check(_lib.xllm_kv_map_pages_many(self._ctx, len(s), s.ctypes.data_as(_i32p), t.ctypes.data_as(_i64p)))
+        s, t = _i32(slots), _i64(min_tokens)
+        self._check(_lib.xllm_kv_map_pages_many(self._ctx, len(s), s.ctypes.data, t.ctypes.data))
 
     def kv_set_len_many(self, slots, kv_lens):
-        s, t = _i32(slots), np.ascontiguousarray(kv_lens, dtype=np.int64)
-        self._check(_lib.xllm_kv_set_len_many(self._ctx, len(s), s.ctypes.data_as(_i32p), t.ctypes.data_as(_i64p)))
+        s, t = _i32(slots), _i64(kv_lens)
+        self._check(_lib.xllm_kv_set_len_many(self._ctx, len(s), s.ctypes.data, t.ctypes.data))
 
     def kv_release(self, slot: int, mode: int = 0):
         self._check(_lib.xllm_kv_release(self._ctx, slot, mode))
@@ -234,8 +242,8 @@ class Context:
     # -- KV writes --
     def kv_append(self, slots, n_new, k_new, v_new, stream=None):
         s, n = _i32(slots), _i32(n_new)
-        self._check(_lib.xllm_kv_append(self._ctx, len(s), s.ctypes.data_as(_i32p), n.ctypes.data_as(_i32p), _ptr(k_new),
-                                        _ptr(v_new), _stream(stream)))
+        self._check(_lib.xllm_kv_append(self._ctx, len(s), s.ctypes.data, n.ctypes.data, _ptr(k_new), _ptr(v_new),
+                                        _stream(stream)))
 
     def kv_gather(self, slot: int, first_token: int, n_tokens: int, k_out, v_out, stream=None):
         self._check(_lib.xllm_kv_gather(self._ctx, slot, first_token, n_tokens, _ptr(k_out), _ptr(v_out), _stream(stream)))
@@ -243,13 +251,13 @@ class Context:
     # -- attention --
     def decode_attention(self, slots, q, out, lse_out=None, scale: float = 1.0, stream=None):
         s = _i32(slots)
-        self._check(_lib.xllm_decode_attention(self._ctx, len(s), s.ctypes.data_as(_i32p), _ptr(q), _ptr(out), _ptr(lse_out),
-                                               scale, _stream(stream)))
+        self._check(_lib.xllm_decode_attention(self._ctx, len(s), s.ctypes.data, _ptr(q), _ptr(out), _ptr(lse_out), scale,
+                                               _stream(stream)))
 
     def verify_attention(self, slots, q_lens, q, out, lse_out=None, scale: float = 1.0, stream=None):
         s, ql = _i32(slots), _i32(q_lens)
-        self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data_as(_i32p), ql.ctypes.data_as(_i32p), _ptr(q),
-                                               _ptr(out), _ptr(lse_out), scale, _stream(stream)))
+        self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(q), _ptr(out),
+                                               _ptr(lse_out), scale, _stream(stream)))
 
     def sync_check(self, stream=None):
         self._check(_lib.xllm_sync_check(self._ctx, _stream(stream)))

@@ -39,7 +39,8 @@ struct xllm_ctx {
     std::string err;
     PlanTuning tune;
 
-    // staging ring: pinned host buffers, one device copy target each, one completion event each
+    // staging ring: pinned host buffers mapped into the device address space (kernels read the small work lists in
+    // place, no copy is enqueued), one completion event each
     size_t stage_bytes = 0;
     char *h_stage[kRing] = {};
     char *d_stage[kRing] = {};
@@ -49,6 +50,7 @@ struct xllm_ctx {
     cudaStream_t last_stream = nullptr;
 
     float *d_part_o = nullptr, *d_part_lse = nullptr;
+    int32_t *d_counters = nullptr;  // arrival counters of split units (zero between launches)
     unsigned long long *d_trace = nullptr;  // per-CTA cycle counters, only when XLLM_TRACE is set in the environment
     int32_t max_partials = 0, max_items = 0;
     int32_t *h_error = nullptr, *d_error = nullptr;  // mapped pinned word written by kernels whose waits expired
@@ -62,7 +64,8 @@ struct xllm_ctx {
     xllm_stats st{};
 
     std::vector<xllm_work_item> items;
-    std::vector<int32_t> cta_begin;
+    std::vector<int32_t> cta_begin, q_row0, part_first, part_count;
+    std::vector<CombineDesc> combine;
     std::vector<int64_t> kv_lens;
     std::vector<uint8_t> seen;
 };
@@ -83,6 +86,9 @@ xllm_status check_device_flag(xllm_ctx *ctx) {
     if (ctx->h_error && *reinterpret_cast<volatile int32_t *>(ctx->h_error) != 0) {
         const int code = *ctx->h_error;
         *ctx->h_error = 0;
+        // the launch that gave up may have left arrival counters of split units behind
+        cudaDeviceSynchronize();
+        if (ctx->d_counters) cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * (size_t)ctx->max_partials);
         return fail(ctx, XLLM_ERR_CUDA, "attention kernel: a bounded device-side wait expired (code " + std::to_string(code) +
                                             "); the results of that launch are invalid");
     }
@@ -205,10 +211,11 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     if (n_items > ctx->max_items || n_partials > ctx->max_partials)
         return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": work list exceeds the workspace sized at init");
 
-    // split units -> combine descriptors (a unit's partials are consecutive)
-    std::vector<CombineDesc> combine;
+    // split units: a unit's pieces have consecutive partial slots.  Units in few pieces are merged by the attention
+    // kernel itself (the piece that finishes last does it); the others go to the combine kernel.
     const int32_t G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
-    std::vector<int32_t> q_row0((size_t)n_req);
+    std::vector<int32_t> &q_row0 = ctx->q_row0;
+    q_row0.resize((size_t)n_req);
     {
         int32_t acc = 0;
         for (int32_t i = 0; i < n_req; ++i) {
@@ -216,14 +223,27 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
             acc += q_lens ? q_lens[i] : 1;
         }
     }
-    int32_t last_unit = -1;
-    for (const xllm_work_item &it : ctx->items) {
-        if (it.partial_idx < 0) continue;
-        if (it.unit == last_unit) {
-            ++combine.back().n_parts;
-        } else {
-            combine.push_back({it.partial_idx, 1, q_row0[(size_t)it.req] + it.q_tok0, it.kv_head * G + it.g0, it.n_q_tok, it.n_g});
-            last_unit = it.unit;
+    std::vector<int32_t> &part_first = ctx->part_first, &part_count = ctx->part_count;  // indexed by partial slot
+    part_first.assign((size_t)n_partials, 0);
+    part_count.assign((size_t)n_partials, 0);
+    std::vector<CombineDesc> &combine = ctx->combine;
+    combine.clear();
+    {
+        int32_t last_unit = -1, first = 0;
+        for (const xllm_work_item &it : ctx->items) {
+            if (it.partial_idx < 0) continue;
+            if (it.unit != last_unit) {
+                last_unit = it.unit;
+                first = it.partial_idx;
+            }
+            part_first[(size_t)it.partial_idx] = first;
+            ++part_count[(size_t)first];
+        }
+        for (const xllm_work_item &it : ctx->items) {
+            if (it.partial_idx < 0 || part_first[(size_t)it.partial_idx] != it.partial_idx) continue;  // first piece only
+            if (part_count[(size_t)it.partial_idx] > kFuseMaxParts)
+                combine.push_back({it.partial_idx, part_count[(size_t)it.partial_idx], q_row0[(size_t)it.req] + it.q_tok0,
+                                   it.kv_head * G + it.g0, it.n_q_tok, it.n_g});
         }
     }
 
@@ -251,13 +271,15 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         di[i].head0 = (int16_t)(w.kv_head * G + w.g0);
         di[i].n_q_tok = (uint8_t)w.n_q_tok;
         di[i].n_g = (uint8_t)w.n_g;
+        di[i].part_first = w.partial_idx >= 0 ? part_first[(size_t)w.partial_idx] : 0;
+        const int32_t pieces = w.partial_idx >= 0 ? part_count[(size_t)di[i].part_first] : 0;
+        di[i].n_parts = pieces <= kFuseMaxParts ? pieces : 0;
+        di[i].pad[0] = di[i].pad[1] = 0;
     }
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    char *d = ctx->d_stage[idx];
-    e = (int)cudaMemcpyAsync(d, h, total, cudaMemcpyHostToDevice, stream);
-    if (e) return cuda_fail(ctx, "staging the work list", e);
+    char *d = ctx->d_stage[idx];  // the same bytes seen from the device (mapped pinned memory)
 
     AttnLaunch al{};
     al.items = reinterpret_cast<const DevItem *>(d + off_items);
@@ -266,6 +288,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.lse_out = lse_out;
     al.part_o = ctx->d_part_o;
     al.part_lse = ctx->d_part_lse;
+    al.counters = ctx->d_counters;
     al.error_flag = ctx->d_error;
     al.trace = ctx->d_trace;
     al.n_q_heads = ctx->cfg.n_q_heads;
@@ -274,6 +297,8 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.scale_log2 = scale * 1.4426950408889634f;
     al.n_ctas = ctx->sm_count;
     std::memcpy(al.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    for (int32_t c = 0; c < ctx->sm_count; ++c)
+        if (al.cta_begin[c] < al.cta_begin[c + 1]) al.first_item[c] = di[al.cta_begin[c]];
     time_begin(ctx, 0, stream);
     e = launch_attention(al, stream);
     time_end(ctx, stream);
@@ -372,12 +397,14 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     if (!ctx->host_only) {
         cudaError_t e = cudaSuccess;
         for (int i = 0; i < kRing && e == cudaSuccess; ++i) {
-            e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_stage[i]), ctx->stage_bytes, cudaHostAllocDefault);
-            if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_stage[i]), ctx->stage_bytes);
+            e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_stage[i]), ctx->stage_bytes, cudaHostAllocMapped);
+            if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&ctx->d_stage[i]), ctx->h_stage[i], 0);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->done[i], cudaEventDisableTiming);
         }
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * kMaxRows * cfg->head_dim);
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * kMaxRows);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_counters), sizeof(int32_t) * (size_t)ctx->max_partials);
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * (size_t)ctx->max_partials);
         if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_error), sizeof(int32_t), cudaHostAllocMapped);
         if (e == cudaSuccess) {
             *ctx->h_error = 0;
@@ -411,11 +438,11 @@ xllm_status xllm_shutdown(xllm_ctx *ctx) {
     if (!ctx->host_only) {
         for (int i = 0; i < kRing; ++i) {
             if (ctx->h_stage[i]) cudaFreeHost(ctx->h_stage[i]);
-            if (ctx->d_stage[i]) cudaFree(ctx->d_stage[i]);
             if (ctx->done[i]) cudaEventDestroy(ctx->done[i]);
         }
         if (ctx->d_part_o) cudaFree(ctx->d_part_o);
         if (ctx->d_part_lse) cudaFree(ctx->d_part_lse);
+        if (ctx->d_counters) cudaFree(ctx->d_counters);
         if (ctx->d_trace) cudaFree(ctx->d_trace);
         if (ctx->h_error) cudaFreeHost(ctx->h_error);
         for (TimedLaunch &t : ctx->timed) {
@@ -597,8 +624,6 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         row0 += n_new[i];
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    e = (int)cudaMemcpyAsync(ctx->d_stage[idx], ad, sizeof(AppendDesc) * (size_t)n_desc, cudaMemcpyHostToDevice, stream);
-    if (e) return cuda_fail(ctx, "staging the append list", e);
     time_begin(ctx, 2, stream);
     e = launch_append(reinterpret_cast<const AppendDesc *>(ctx->d_stage[idx]), n_desc, max_new, k_new, v_new,
                       ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);

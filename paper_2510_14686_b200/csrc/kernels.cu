@@ -20,6 +20,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <utility>
 
 #include "xllm_internal.h"
 
@@ -65,8 +66,8 @@ struct Cfg {
     static constexpr int kOffQ = kOffP + 2 * 2 * kMaxRows * kPPitch;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
     static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(DevItem);
-    static constexpr int kNumBars = 2 * kHalfStages + 6;
-    static constexpr int kOffFlags = kOffBars + kNumBars * 8;
+    static constexpr int kNumBars = 2 * kHalfStages + 7;
+    static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast
     static constexpr int kSmemBytes = kOffFlags + 16;
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
@@ -144,6 +145,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+
+// Programmatic dependent launch: every kernel of the library is launched so that its blocks may become resident
+// while the previous kernel of the stream drains.  Nothing that kernel wrote (and nothing it may still read) is
+// touched before grid_dependency_wait(), which returns once the previous kernel has completed and flushed.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void group_bar(int group) {
     __syncwarp();  // the barrier instruction is warp-aligned: make sure the lanes have re-converged
@@ -318,6 +325,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const uint32_t bar_qempty = bar_qfull + 16;                       // [2] query rows loaded to registers (8 warps)
     const uint32_t bar_mfull = bar_qempty + 16;                       // group states of an item written (8 warps)
     const uint32_t bar_mempty = bar_mfull + 8;                        // ... and read by the epilogue (3 warps)
+    const uint32_t bar_items = bar_mempty + 8;                        // first batch of item records is in shared memory
     const unsigned long long t_start = TRACE ? clock64() : 0ull;
     const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
 
@@ -333,6 +341,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         }
         mbar_init(bar_mfull, kConsumerWarps);
         mbar_init(bar_mempty, kEpilogueWarps);
+        mbar_init(bar_items, kEpilogueWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -342,18 +351,46 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     uint32_t item_seq = 0;  // items started so far
     unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0;
 
+    __syncthreads();          // barriers initialised
+    grid_launch_dependents();  // the next kernel of the stream may start its own prologue
+    grid_dependency_wait();    // from here on q, the KV ranges and the outputs may be touched
+
     for (int batch_lo = item_lo; batch_lo < item_hi; batch_lo += kItemBatch) {
         const int nb = min(kItemBatch, item_hi - batch_lo);
-        if (batch_lo != item_lo) __syncthreads();  // everyone is done with the previous batch's records
-        for (int i = tid; i < nb * 2; i += kThreads)   // 32-byte records moved as 16-byte halves
-            reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
-        __syncthreads();
+        const bool first_batch = batch_lo == item_lo;
+        // Item records live in host memory mapped into the device: fetching them costs a trip over PCIe.  In the
+        // first batch the record of item 0 comes from the kernel parameters and the epilogue warps (idle until the
+        // first item is finished) fetch the rest, so the first loads start at once; later batches (more than
+        // kItemBatch items in a CTA) are fetched by everybody between two CTA-wide barriers.
+        if (first_batch) {
+            if (warp >= kEpilogueWarp0) {
+                for (int i = tid - kEpilogueWarp0 * 32; i < nb * 3; i += kEpilogueThreads)  // 48-byte records, 16-byte pieces
+                    reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_items);
+            }
+        } else {
+            __syncthreads();  // everyone is done with the previous batch's records
+            for (int i = tid; i < nb * 3; i += kThreads)
+                reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
+            __syncthreads();
+        }
+        // record of item i of this batch; waits (once) for the fetch above before the first use of shared memory
+        bool items_ready = !first_batch;
+        auto item_at = [&](int i) -> DevItem {
+            if (first_batch && i == 0) return p.first_item[blockIdx.x];
+            if (!items_ready) {
+                mbar_wait(bar_items, 0, abort_flag, p.error_flag, 8);
+                items_ready = true;
+            }
+            return sitems[i];
+        };
 
         if (warp == kProducerWarp) {
             // ================= producer =================
             if (lane == 0) {
                 for (int i = 0; i < nb; ++i) {
-                    const DevItem it = sitems[i];
+                    const DevItem it = item_at(i);
                     const int n_rows = it.n_q_tok * it.n_g;
                     const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
                     if (mbar_wait(bar_qempty + qb * 8, qph ^ 1, abort_flag, p.error_flag, 1)) {
@@ -385,8 +422,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                         }
                     }
                 }
-            } else {
-                for (int i = 0; i < nb; ++i) fill += sitems[i].tile_end - sitems[i].tile_begin;
             }
             fill = __shfl_sync(0xffffffffu, fill, 0);
         } else if (warp < kConsumerWarps) {
@@ -400,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             const uint32_t p_base = smem_base + C::kOffP + group * (2 * kMaxRows * C::kPPitch);
             uint32_t my_tiles = 0;  // tiles this group has processed: selects the double buffer of maxima / weights
             for (int i = 0; i < nb; ++i) {
-                const DevItem it = sitems[i];
+                const DevItem it = item_at(i);
                 const int n_rows = it.n_q_tok * it.n_g;
                 const int row_limit0 = it.kv_end - it.n_q_tok + 1;
                 const uint32_t seq = item_seq + i, qb = seq & 1, qph = (seq >> 1) & 1;
@@ -497,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             const float *merge_l = reinterpret_cast<const float *>(smem + C::kOffMergeL);
             constexpr int kC4 = D / 4;  // float4 columns per row
             for (int i = 0; i < nb; ++i) {
-                const DevItem it = sitems[i];
+                const DevItem it = item_at(i);
                 const int n_rows = it.n_q_tok * it.n_g;
                 const uint32_t seq = item_seq + i;
                 const bool live = mbar_wait(bar_mfull, seq & 1, abort_flag, p.error_flag, 6);
@@ -531,27 +566,66 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_mempty);
+                if (lane == 0) mbar_arrive(bar_mempty);  // the consumers may overwrite the group states
+                if (live && it.partial_idx >= 0 && it.n_parts > 0) {
+                    // Lightly split unit: whichever piece finishes last merges all pieces (log-sum-exp) and writes the
+                    // final rows, so no second launch is needed.  Release: partial stores, fence, barrier, one atomic.
+                    // Acquire: atomic result, barrier, fence, loads that bypass L1.
+                    volatile int *bcast = reinterpret_cast<volatile int *>(smem + C::kOffFlags) + 1;
+                    __threadfence();
+                    asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");
+                    if (et == 0) *bcast = atomicAdd(p.counters + it.part_first, 1);
+                    asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");
+                    if (*bcast == it.n_parts - 1) {
+                        __threadfence();
+                        for (int idx = et; idx < n_rows * kC4; idx += kEpilogueThreads) {
+                            const int row = idx / kC4, c4 = idx - row * kC4;
+                            float M = -INFINITY;
+                            for (int s2 = 0; s2 < it.n_parts; ++s2)
+                                M = fmaxf(M, __ldcg(p.part_lse + (int64_t)(it.part_first + s2) * kMaxRows + row));
+                            const float Ms = (M == -INFINITY) ? 0.f : M;
+                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                            float W = 0.f;
+                            for (int s2 = 0; s2 < it.n_parts; ++s2) {
+                                const int64_t pi = it.part_first + s2;
+                                const float w = exp2f(__ldcg(p.part_lse + pi * kMaxRows + row) - Ms);  // 0 for a piece without keys
+                                const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.part_o + (pi * kMaxRows + row) * D) + c4);
+                                W += w;
+                                acc.x += w * v.x;
+                                acc.y += w * v.y;
+                                acc.z += w * v.z;
+                                acc.w += w * v.w;
+                            }
+                            const float inv = (W > 0.f) ? 1.f / W : 0.f;
+                            const int ti = row / it.n_g, gi = row - ti * it.n_g;
+                            const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
+                            *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
+                                make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                            if (c4 == 0 && p.lse_out)
+                                p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
+                        }
+                        if (et == 0) p.counters[it.part_first] = 0;  // ready for the next launch
+                    }
+                }
                 if (TRACE) tr_epi += clock64() - t0;
             }
-            for (int i = 0; i < nb; ++i) fill += sitems[i].tile_end - sitems[i].tile_begin;
         }
         item_seq += nb;
     }
 
     // trace layout (16 words per CTA): 0 cycles of warp 0, 1 cycles to its first finished tile, 2 cycles in tile loops
-    // (warp 0), 3 unused, 4 waiting for query rows, 5 item hand-off incl. waiting for the epilogue, 6 items, 7 tiles,
+    // (warp 0), 3 global-timer ns at CTA start (9: at the end of warp 4), 4 waiting for query rows, 5 item hand-off incl. waiting for the epilogue, 6 items, 7 tiles,
     // 8/10 the same as 2/5 for warp 4, 11 producer cycles waiting for free ring slots, 12 producer cycles,
     // 13 epilogue busy cycles, 14 epilogue cycles, 15 nanoseconds of warp 0 (global timer).
     if (TRACE && lane == 0 && (warp == 0 || warp == 4 || warp == kProducerWarp || warp == kEpilogueWarp0)) {
         unsigned long long *tr = p.trace + (int64_t)blockIdx.x * kTraceWords;
         const unsigned long long total = clock64() - t_start;
         if (warp == 0) {
-            tr[0] = total; tr[1] = tr_first; tr[2] = tr_tiles; tr[3] = 0; tr[4] = tr_wait_q; tr[5] = tr_switch;
+            tr[0] = total; tr[1] = tr_first; tr[2] = tr_tiles; tr[3] = g_start; tr[4] = tr_wait_q; tr[5] = tr_switch;
             tr[6] = (unsigned long long)(item_hi - item_lo); tr[7] = fill;
             tr[15] = globaltimer_ns() - g_start;
         } else if (warp == 4) {
-            tr[8] = tr_tiles; tr[9] = 0; tr[10] = tr_switch;
+            tr[8] = tr_tiles; tr[9] = globaltimer_ns(); tr[10] = tr_switch;
         } else if (warp == kProducerWarp) {
             tr[11] = tr_wait_empty; tr[12] = total;
         } else {
@@ -580,6 +654,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 // ---- LSE combine: merge the partial results of every split unit -------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
+    grid_launch_dependents();
+    grid_dependency_wait();  // the partial results come from the attention kernel launched just before
     const CombineDesc d = p.descs[blockIdx.x];
     const int row = blockIdx.y;
     if (row >= d.n_q_tok * d.n_g) return;
@@ -616,6 +692,8 @@ __device__ __forceinline__ int64_t slot_chunk_offset(int64_t pos, int h, int whi
 
 __global__ void append_kernel(const AppendDesc *__restrict__ descs, const uint4 *__restrict__ k_new,
                               const uint4 *__restrict__ v_new, int n_kv_heads, int D) {
+    grid_launch_dependents();
+    grid_dependency_wait();  // the previous kernel may still read the slots or write k_new / v_new
     const AppendDesc d = descs[blockIdx.y];
     const int cpr = D / 8;                       // chunks per head row
     const int row_chunks = n_kv_heads * cpr;     // chunks per token of one tensor
@@ -633,6 +711,8 @@ __global__ void append_kernel(const AppendDesc *__restrict__ descs, const uint4 
 
 __global__ void gather_kernel(uint64_t base, int64_t first_token, int64_t n_tokens, uint4 *__restrict__ k_out,
                               uint4 *__restrict__ v_out, int n_kv_heads, int D) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int cpr = D / 8;
     const int64_t per_tensor = n_tokens * n_kv_heads * cpr;
     const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -665,26 +745,40 @@ int configure_kernels(int32_t head_dim) {
     return (int)e;
 }
 
+// Launch with the programmatic-stream-serialization attribute (see grid_dependency_wait above).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 int launch_attention(const AttnLaunch &p, void *stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
     if (p.head_dim == 128) {
-        if (p.trace) attention_kernel<128, true><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
-        else attention_kernel<128, false><<<p.n_ctas, kThreads, Cfg<128>::kSmemBytes, st>>>(p);
+        if (p.trace) e = launch_pdl(attention_kernel<128, true>, dim3(p.n_ctas), dim3(kThreads), Cfg<128>::kSmemBytes, st, p);
+        else e = launch_pdl(attention_kernel<128, false>, dim3(p.n_ctas), dim3(kThreads), Cfg<128>::kSmemBytes, st, p);
     } else {
-        if (p.trace) attention_kernel<64, true><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
-        else attention_kernel<64, false><<<p.n_ctas, kThreads, Cfg<64>::kSmemBytes, st>>>(p);
+        if (p.trace) e = launch_pdl(attention_kernel<64, true>, dim3(p.n_ctas), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
+        else e = launch_pdl(attention_kernel<64, false>, dim3(p.n_ctas), dim3(kThreads), Cfg<64>::kSmemBytes, st, p);
     }
-    return (int)cudaGetLastError();
+    return (int)e;
 }
 
 int launch_combine(const CombineLaunch &p, void *stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     dim3 grid(p.n_units, kMaxRows);
-    if (p.head_dim == 128)
-        combine_kernel<128><<<grid, 128, 0, st>>>(p);
-    else
-        combine_kernel<64><<<grid, 64, 0, st>>>(p);
-    return (int)cudaGetLastError();
+    if (p.head_dim == 128) return (int)launch_pdl(combine_kernel<128>, grid, dim3(128), 0, st, p);
+    return (int)launch_pdl(combine_kernel<64>, grid, dim3(64), 0, st, p);
 }
 
 int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *k_new, const void *v_new,
@@ -693,9 +787,8 @@ int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const
     const int threads = 256;
     const int64_t bx = std::min<int64_t>((per_req + threads - 1) / threads, 4096);
     dim3 grid((unsigned)bx, (unsigned)n_req);
-    append_kernel<<<grid, threads, 0, static_cast<cudaStream_t>(stream)>>>(
-        descs, static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), n_kv_heads, head_dim);
-    return (int)cudaGetLastError();
+    return (int)launch_pdl(append_kernel, grid, dim3(threads), 0, static_cast<cudaStream_t>(stream), descs,
+                           static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), (int)n_kv_heads, (int)head_dim);
 }
 
 int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,
@@ -703,9 +796,9 @@ int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_
     const int64_t total = 2 * n_tokens * n_kv_heads * (head_dim / 8);
     const int threads = 256;
     const int64_t blocks = (total + threads - 1) / threads;
-    gather_kernel<<<(unsigned)blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
-        base, first_token, n_tokens, static_cast<uint4 *>(k_out), static_cast<uint4 *>(v_out), n_kv_heads, head_dim);
-    return (int)cudaGetLastError();
+    return (int)launch_pdl(gather_kernel, dim3((unsigned)blocks), dim3(threads), 0, static_cast<cudaStream_t>(stream), base,
+                           first_token, n_tokens, static_cast<uint4 *>(k_out), static_cast<uint4 *>(v_out), (int)n_kv_heads,
+                           (int)head_dim);
 }
 
 }  // namespace xllm

@@ -21,9 +21,8 @@ struct Unit {
     int16_t q_tok0, n_q_tok, g0, n_g;
     int32_t n_tiles;  // tiles that hold keys visible to the unit's last row
     int32_t max_cut;  // largest tile boundary at which a split may start so that the first row still sees a key
-};
-struct Cut {
-    int32_t unit, tile;
+    int32_t last_cost;  // cost of the last (possibly short) tile
+    int32_t overhead;   // fixed cost of the unit: query load, hand-off to the epilogue, output rows
 };
 }  // namespace
 
@@ -47,7 +46,7 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
                     const int64_t vis_last = kv - ql + t0 + nt;  // keys visible to the last row
                     const int64_t vis_first = kv - ql + t0 + 1;  // keys visible to the first row
                     Unit u{r, h, (int16_t)t0, (int16_t)nt, 0, (int16_t)G, (int32_t)((vis_last + T - 1) / T),
-                           (int32_t)((vis_first - 1) / T)};
+                           (int32_t)((vis_first - 1) / T), 0, 0};
                     units.push_back(u);
                 }
             } else {
@@ -55,7 +54,7 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
                     const int64_t vis = kv - ql + t0 + 1;
                     for (int32_t g0 = 0; g0 < G; g0 += kMaxRows) {
                         Unit u{r, h, (int16_t)t0, 1, (int16_t)g0, (int16_t)std::min(kMaxRows, G - g0),
-                               (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T)};
+                               (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T), 0, 0};
                         units.push_back(u);
                     }
                 }
@@ -63,64 +62,81 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
         }
     }
     const int32_t U = static_cast<int32_t>(units.size());
-    // cost axis: start position of every unit
+    // cost axis: start position of every unit.  A full tile costs tile_cost; the last tile of a unit is fetched
+    // in 16-token steps: half of its cost is fixed, half goes with the volume; a unit's fixed cost grows with its row count.
     std::vector<int64_t> start(static_cast<size_t>(U) + 1);
     start[0] = 0;
-    for (int32_t u = 0; u < U; ++u)
-        start[u + 1] = start[u] + tune.unit_overhead + (int64_t)tune.tile_cost * units[u].n_tiles;
-    const int64_t total = start[U];
-
-    std::vector<Cut> cuts(static_cast<size_t>(n_ctas) + 1);
-    cuts[0] = {0, 0};
-    cuts[n_ctas] = {U, 0};
-    int32_t u = 0;
-    for (int32_t c = 1; c < n_ctas; ++c) {
-        const int64_t pos = (total * c) / n_ctas;
-        while (u < U && start[u + 1] <= pos) ++u;
-        if (u >= U) {
-            cuts[c] = {U, 0};
-            continue;
-        }
-        const Unit &un = units[u];
-        int64_t b = (pos - start[u] - tune.unit_overhead + tune.tile_cost / 2) / tune.tile_cost;  // nearest tile
-        if (pos - start[u] < tune.unit_overhead) b = 0;
-        b = std::max<int64_t>(0, std::min<int64_t>(b, un.n_tiles));
-        if (b > un.max_cut) b = un.max_cut;                      // every row of a piece must see a key
-        if (b < tune.min_piece_tiles) b = 0;                     // no sliver at the front ...
-        else if (un.n_tiles - b < tune.min_piece_tiles) b = un.n_tiles;  // ... nor at the back
-        Cut cut = (b >= un.n_tiles) ? Cut{u + 1, 0} : Cut{u, (int32_t)b};
-        // cuts never move backwards
-        const Cut &prev = cuts[c - 1];
-        if (cut.unit < prev.unit || (cut.unit == prev.unit && cut.tile < prev.tile)) cut = prev;
-        cuts[c] = cut;
+    for (int32_t u = 0; u < U; ++u) {
+        Unit &un = units[u];
+        const int64_t vis_last = kv_lens[un.req] - (q_lens ? q_lens[un.req] : 1) + un.q_tok0 + un.n_q_tok;
+        const int32_t tail_rows = (int32_t)std::min<int64_t>(T, ((vis_last - (int64_t)(un.n_tiles - 1) * T) + 15) / 16 * 16);
+        un.last_cost = tune.tile_cost / 2 + tune.tile_cost * tail_rows / (2 * T);  // half fixed, half by volume
+        un.overhead = tune.unit_overhead + tune.row_overhead * un.n_q_tok * un.n_g / kMaxRows;
+        start[u + 1] = start[u] + un.overhead + (int64_t)tune.tile_cost * (un.n_tiles - 1) + un.last_cost;
     }
-
+    // Walk the axis once, CTA by CTA.  Each CTA aims at an equal share of what is still to be done; "what is
+    // still to be done" includes the fixed cost a unit's continuation pays again when a cut splits the unit, so the
+    // shares stay equal although every split adds work.
     items.clear();
     cta_begin.assign(static_cast<size_t>(n_ctas) + 1, 0);
     int32_t n_partials = 0;
+    int32_t u = 0, tile = 0;  // next work: unit u from tile `tile` on
+    int64_t mean_overhead = 0;
+    for (const Unit &un : units) mean_overhead += un.overhead;
+    mean_overhead = U ? mean_overhead / U : 0;
+    auto tiles_cost = [&](const Unit &un, int32_t from, int32_t to) -> int64_t {  // cost of tiles [from, to)
+        if (to <= from) return 0;
+        int64_t c = (int64_t)tune.tile_cost * (to - from);
+        if (to == un.n_tiles) c += un.last_cost - tune.tile_cost;
+        return c;
+    };
     for (int32_t c = 0; c < n_ctas; ++c) {
         cta_begin[c] = static_cast<int32_t>(items.size());
-        Cut a = cuts[c];
-        const Cut b = cuts[c + 1];
-        while (a.unit < U && (a.unit < b.unit || (a.unit == b.unit && a.tile < b.tile))) {
-            const Unit &un = units[a.unit];
-            const int32_t te = (a.unit == b.unit) ? b.tile : un.n_tiles;
-            if (te > a.tile) {
-                xllm_work_item it;
-                it.req = un.req;
-                it.kv_head = un.kv_head;
-                it.tile_begin = a.tile;
-                it.tile_end = te;
-                it.q_tok0 = un.q_tok0;
-                it.n_q_tok = un.n_q_tok;
-                it.g0 = un.g0;
-                it.n_g = un.n_g;
-                it.partial_idx = (a.tile == 0 && te == un.n_tiles) ? -1 : n_partials++;
-                it.unit = a.unit;
-                items.push_back(it);
+        if (u >= U) continue;
+        int64_t remaining = start[U] - start[u + 1] + units[u].overhead + tiles_cost(units[u], tile, units[u].n_tiles);
+        remaining += (int64_t)(n_ctas - c - 1) * mean_overhead;  // most of the cuts still to come will split a unit
+        const int64_t target = (c == n_ctas - 1) ? INT64_MAX : (remaining + (n_ctas - c) / 2) / (n_ctas - c);
+        int64_t load = 0;
+        while (u < U) {
+            const Unit &un = units[u];
+            const int32_t left = un.n_tiles - tile;
+            const int64_t whole = un.overhead + tiles_cost(un, tile, un.n_tiles);
+            int32_t take;
+            if (target == INT64_MAX || load + whole <= target + tune.tile_cost / 2) {
+                take = left;  // the rest of the unit fits
+            } else {
+                const int64_t room = target - load - un.overhead;
+                take = room <= 0 ? 0 : (int32_t)std::min<int64_t>(left, (room + tune.tile_cost / 2) / tune.tile_cost);
+                if (tile + take > un.max_cut) take = std::max(0, un.max_cut - tile);  // every row of the next piece must see a key
+                if (left - take < tune.min_piece_tiles) take = (left - take <= take || load == 0) ? left : std::max(0, left - tune.min_piece_tiles);
+                if (take < tune.min_piece_tiles && take < left) take = 0;              // no sliver: leave the unit to the next CTA
+                if (tile + take > un.max_cut && take < left) take = 0;
+                if (take == 0 && load == 0) {  // a CTA with work left must take something: progress is guaranteed
+                    take = std::min(left, std::max(tune.min_piece_tiles, 1));
+                    if (tile + take > un.max_cut) take = left;
+                }
             }
-            if (a.unit == b.unit) break;
-            a = {a.unit + 1, 0};
+            if (take == 0) break;
+            xllm_work_item it;
+            it.req = un.req;
+            it.kv_head = un.kv_head;
+            it.tile_begin = tile;
+            it.tile_end = tile + take;
+            it.q_tok0 = un.q_tok0;
+            it.n_q_tok = un.n_q_tok;
+            it.g0 = un.g0;
+            it.n_g = un.n_g;
+            it.partial_idx = (tile == 0 && take == un.n_tiles) ? -1 : n_partials++;
+            it.unit = u;
+            items.push_back(it);
+            load += un.overhead + tiles_cost(un, tile, tile + take);
+            tile += take;
+            if (tile == un.n_tiles) {
+                ++u;
+                tile = 0;
+            } else {
+                break;  // the unit continues in the next CTA
+            }
         }
     }
     cta_begin[n_ctas] = static_cast<int32_t>(items.size());

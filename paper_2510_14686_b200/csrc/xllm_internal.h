@@ -11,9 +11,11 @@ namespace xllm {
 constexpr int32_t kMaxRows = 16;  // query rows (heads of a GQA group x query tokens) one work item carries
 
 struct PlanTuning {
-    int32_t tile_cost = 4;        // cost of one KV tile block on the partition axis
-    int32_t unit_overhead = 3;    // fixed cost of starting a unit (Q load, merge, output), same scale
-    int32_t min_piece_tiles = 4;  // pieces of a split unit are at least this many tiles
+    // Measured on B200 (per-CTA timers): a work item costs about as much as 1 tile with 4 rows and 2 tiles with 16.
+    int32_t tile_cost = 8;        // cost of one full KV tile block on the partition axis
+    int32_t unit_overhead = 6;    // fixed cost of starting a unit (Q load, hand-off, output), same scale ...
+    int32_t row_overhead = 8;     // ... plus this much for a full 16-row unit, in proportion to its rows
+    int32_t min_piece_tiles = 2;  // pieces of a split unit are at least this many tiles
 };
 
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
@@ -34,7 +36,9 @@ inline int64_t tile_block_bytes(int32_t n_kv_heads, int32_t head_dim) { return n
 // ---- device-side records ------------------------------------------------------------------------------
 constexpr int32_t kMaxCtas = 160;  // upper bound on the persistent grid (B200: 148 SMs)
 
-struct DevItem {            // one work item, resolved on the host against the slot table (32 bytes)
+constexpr int32_t kFuseMaxParts = 8;  // units split into at most this many pieces are merged inside the attention kernel
+
+struct DevItem {            // one work item, resolved on the host against the slot table (48 bytes)
     uint64_t kv;            // address of the item's KV head inside tile block 0 of the slot's range
     int32_t q_row;          // first row of the item's query group in q / out  (request row + q_tok0)
     int32_t partial_idx;    // -1: writes the final output; else slot in the partial workspace
@@ -42,8 +46,11 @@ struct DevItem {            // one work item, resolved on the host against the s
     int32_t kv_end;         // keys visible to the group's last query token
     int16_t head0;          // first query head of the group (kv_head * G + g0)
     uint8_t n_q_tok, n_g;   // rows = n_q_tok * n_g <= kMaxRows
+    int32_t part_first;     // partial slot of the unit's first piece (also the index of the unit's arrival counter)
+    int32_t n_parts;        // pieces of the unit if the last piece to finish merges them in-kernel; 0 = combine kernel
+    int32_t pad[2];
 };
-static_assert(sizeof(DevItem) == 32, "DevItem layout");
+static_assert(sizeof(DevItem) == 48, "DevItem layout");
 
 struct CombineDesc {        // one per split unit
     int32_t partial_begin, n_parts;
@@ -67,12 +74,14 @@ struct AttnLaunch {
     float *lse_out;               // may be null
     float *part_o;                // [n_partials][kMaxRows][D] fp32
     float *part_lse;              // [n_partials][kMaxRows]    (log2 domain)
+    int32_t *counters;            // [n_partials] arrival counters of split units, zero between launches
     int32_t *error_flag;          // host-mapped; set non-zero when a bounded wait expires
     unsigned long long *trace;    // optional per-CTA cycle counters (debug), may be null
     int32_t n_q_heads, n_kv_heads, head_dim;
     float scale_log2;             // scale * log2(e)
     int32_t n_ctas;
     int32_t cta_begin[kMaxCtas + 1];  // CTA c owns items [cta_begin[c], cta_begin[c+1])
+    DevItem first_item[kMaxCtas];     // copy of items[cta_begin[c]]: the first loads need no trip to the item list
 };
 
 struct CombineLaunch {

@@ -100,6 +100,22 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's device time (every rank runs its own replica)."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(tokens_per_step_per_rank: int, world: int, steps: int, ms: float) -> float:
+    """Whole-job KV tokens/s: all ranks' tokens over the slowest rank's time."""
+    return tokens_per_step_per_rank * world * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------------------------
 # reference arm: the oracle as it stands, on host cores, bounded sample per step
 # ------------------------------------------------------------------------------------------------------------
@@ -272,12 +288,7 @@ def run_ours(args):
             fn(first + i)
         ev1.record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
 
     for i in range(max(args.warmup, 3)):
         rep.step(i)
@@ -323,8 +334,8 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peak()
-    value = tokens_per_step * world * args.steps / (ms * 1e-3)
-    e2e_value = tokens_per_step * world * args.steps / (ms_e2e * 1e-3)
+    value = job_throughput(tokens_per_step, world, args.steps, ms)
+    e2e_value = job_throughput(tokens_per_step, world, args.steps, ms_e2e)
     achieved = alg_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
     h2d = int(rep.h_q.numel() + rep.h_k.numel() + rep.h_v.numel()) * 2
     d2h = int(rep.h_out.numel()) * 2

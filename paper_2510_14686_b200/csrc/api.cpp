@@ -375,6 +375,15 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         drv = make_cuda_driver(&derr);
         if (!drv) return bad(XLLM_ERR_CUDA, derr);
     }
+    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece": planner cost model override (tuning aid)
+        int a, b, c, d;
+        if (std::sscanf(t, "%d,%d,%d,%d", &a, &b, &c, &d) == 4 && a > 0 && b >= 0 && c >= 0 && d >= 1) {
+            ctx->tune.tile_cost = a;
+            ctx->tune.unit_overhead = b;
+            ctx->tune.row_overhead = c;
+            ctx->tune.min_piece_tiles = d;
+        }
+    }
     ctx->xt.reset(new XTensor(std::move(drv), cfg->device, cfg->max_slots, cfg->max_seq_len, row_bytes));
     std::string perr;
     xllm_status st = ctx->xt->init_pool(cfg->phys_budget_bytes, cfg->page_bytes, (cfg->flags & XLLM_FLAG_LAZY_PAGES) != 0, &perr);
@@ -625,11 +634,11 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     time_begin(ctx, 2, stream);
-    e = launch_append(reinterpret_cast<const AppendDesc *>(ctx->d_stage[idx]), n_desc, max_new, k_new, v_new,
+    e = launch_append(ad, n_desc, max_new, k_new, v_new,
                       ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);
     time_end(ctx, stream);
     if (e) return cuda_fail(ctx, "launching the append kernel", e);
-    ++ctx->st.kernel_launches;
+    ctx->st.kernel_launches += (n_desc + kAppendBatch - 1) / kAppendBatch;
     finish_launch(ctx, idx, stream);
     for (int32_t i = 0; i < n_req; ++i) {
         SlotRecord &s = ctx->xt->slot(slots[i]);

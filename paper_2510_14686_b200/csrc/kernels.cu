@@ -690,11 +690,11 @@ __device__ __forceinline__ int64_t slot_chunk_offset(int64_t pos, int h, int whi
            (int64_t)which * (panels * kPanelBytes) + (c >> 3) * kPanelBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
 }
 
-__global__ void append_kernel(const AppendDesc *__restrict__ descs, const uint4 *__restrict__ k_new,
+__global__ void append_kernel(const __grid_constant__ AppendLaunch descs, const uint4 *__restrict__ k_new,
                               const uint4 *__restrict__ v_new, int n_kv_heads, int D) {
     grid_launch_dependents();
     grid_dependency_wait();  // the previous kernel may still read the slots or write k_new / v_new
-    const AppendDesc d = descs[blockIdx.y];
+    const AppendDesc d = descs.d[blockIdx.y];
     const int cpr = D / 8;                       // chunks per head row
     const int row_chunks = n_kv_heads * cpr;     // chunks per token of one tensor
     const int64_t per_tensor = (int64_t)d.n_new * row_chunks;
@@ -786,9 +786,17 @@ int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const
     const int64_t per_req = 2ll * max_new * n_kv_heads * (head_dim / 8);  // chunks of the largest request
     const int threads = 256;
     const int64_t bx = std::min<int64_t>((per_req + threads - 1) / threads, 4096);
-    dim3 grid((unsigned)bx, (unsigned)n_req);
-    return (int)launch_pdl(append_kernel, grid, dim3(threads), 0, static_cast<cudaStream_t>(stream), descs,
-                           static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), (int)n_kv_heads, (int)head_dim);
+    for (int32_t first = 0; first < n_req; first += kAppendBatch) {  // descriptors go by value: no trip to host memory
+        const int32_t n = std::min(kAppendBatch, n_req - first);
+        AppendLaunch al;
+        for (int32_t i = 0; i < n; ++i) al.d[i] = descs[first + i];
+        dim3 grid((unsigned)bx, (unsigned)n);
+        const cudaError_t e = launch_pdl(append_kernel, grid, dim3(threads), 0, static_cast<cudaStream_t>(stream), al,
+                                         static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), (int)n_kv_heads,
+                                         (int)head_dim);
+        if (e != cudaSuccess) return (int)e;
+    }
+    return 0;
 }
 
 int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,

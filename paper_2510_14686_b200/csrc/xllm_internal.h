@@ -15,7 +15,7 @@ struct PlanTuning {
     int32_t tile_cost = 8;        // cost of one full KV tile block on the partition axis
     int32_t unit_overhead = 6;    // fixed cost of starting a unit (Q load, hand-off, output), same scale ...
     int32_t row_overhead = 8;     // ... plus this much for a full 16-row unit, in proportion to its rows
-    int32_t min_piece_tiles = 2;  // pieces of a split unit are at least this many tiles
+    int32_t min_piece_tiles = 6;  // pieces of a split unit are at least this many tiles (swept on B200: 4..8 are within noise)
 };
 
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
@@ -65,6 +65,11 @@ struct AppendDesc {         // one per request of an append call
     int32_t row0;           // first source row
     int32_t n_new;
     int32_t pad;
+};
+
+constexpr int32_t kAppendBatch = 128;  // requests per append launch (their descriptors travel as kernel parameters)
+struct AppendLaunch {
+    AppendDesc d[kAppendBatch];
 };
 
 struct AttnLaunch {

@@ -81,9 +81,9 @@ def test_named_workloads(binding, name):
     items, loads, n_parts = check_plan(binding, kv, ql, s.n_q_heads, s.n_kv_heads, 148)
     total = loads.sum()
     if name != "tiny":
-        # near-equal cost per CTA (slack: the no-sliver rule may move a cut by a few tiles)
-        assert loads.max() - total / 148 <= 8 * 4, (loads.max(), total / 148, loads.min())
-        assert total / 148 - loads[:-1].min() <= 8 * 6, (loads.min(), total / 148)
+        # near-equal cost per CTA (slack: the no-sliver rule moves a cut by up to min_piece_tiles = 6 tiles)
+        assert loads.max() - total / 148 <= 8 * 7, (loads.max(), total / 148, loads.min())
+        assert total / 148 - loads[:-1].min() <= 8 * 12, (loads.min(), total / 148)
         assert n_parts <= 2 * 148
 
 

@@ -15,25 +15,58 @@
 
 namespace xllm {
 
-namespace {
-struct Unit {
-    int32_t req, kv_head;
-    int16_t q_tok0, n_q_tok, g0, n_g;
-    int32_t n_tiles;  // tiles that hold keys visible to the unit's last row
-    int32_t max_cut;  // largest tile boundary at which a split may start so that the first row still sees a key
-    int32_t last_cost;  // cost of the last (possibly short) tile
-    int32_t overhead;   // fixed cost of the unit: query load, hand-off to the epilogue, output rows
-};
-}  // namespace
+using Unit = PlanUnit;
+
+int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads) {
+    if (n_req < 1 || n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads) return -1;
+    const int32_t G = n_q_heads / n_kv_heads;
+    int64_t n = 0;
+    for (int32_t r = 0; r < n_req; ++r) {
+        const int32_t ql = q_lens ? q_lens[r] : 1;
+        if (ql < 1) return -1;
+        const int32_t per = std::max(1, kMaxRows / G);
+        n += (G <= kMaxRows) ? (int64_t)n_kv_heads * ((ql + per - 1) / per) : (int64_t)n_kv_heads * ql * ((G + kMaxRows - 1) / kMaxRows);
+    }
+    return n;
+}
 
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
                    std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out) {
+    const int64_t n_units = plan_count_units(n_req, q_lens, n_q_heads, n_kv_heads);
+    if (n_units < 0 || n_ctas < 1 || n_units > INT32_MAX / 2) return -1;
+    std::vector<PlanUnit> units((size_t)n_units);
+    std::vector<int64_t> start((size_t)n_units + 1);
+    items.resize((size_t)n_units + (size_t)n_ctas);
+    cta_begin.assign((size_t)n_ctas + 1, 0);
+    PlanBuffers buf{units.data(), start.data(), (int32_t)n_units, items.data(), (int32_t)items.size(), cta_begin.data()};
+    int32_t n_items = 0;
+    const int rc = plan_partition_core(n_req, kv_lens, q_lens, n_q_heads, n_kv_heads, n_ctas, tune, buf, &n_items, n_units_out,
+                                       n_partials_out);
+    items.resize(rc == 0 ? (size_t)n_items : 0);
+    return rc;
+}
+
+// The planner proper.  Works in caller-provided arrays and allocates nothing; returns -1 for bad sizes, -2 when an
+// array is too small.
+int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads,
+                        int32_t n_ctas, const PlanTuning &tune, const PlanBuffers &buf, int32_t *n_items_out,
+                        int32_t *n_units_out, int32_t *n_partials_out) {
     if (n_req < 1 || n_ctas < 1 || n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads) return -1;
     const int32_t G = n_q_heads / n_kv_heads;
     const int32_t T = XLLM_TILE_TOKENS;
-    std::vector<Unit> units;
-    units.reserve(static_cast<size_t>(n_req) * n_kv_heads);
+    struct UnitList {  // push_back into the caller's array
+        PlanUnit *p;
+        int32_t n, cap;
+        bool overflow;
+        void push_back(const PlanUnit &u) {
+            if (n < cap) p[n++] = u; else overflow = true;
+        }
+        PlanUnit &operator[](int32_t i) { return p[i]; }
+        size_t size() const { return (size_t)n; }
+        PlanUnit *begin() { return p; }
+        PlanUnit *end() { return p + n; }
+    } units{buf.units, 0, buf.cap_units, false};
     for (int32_t r = 0; r < n_req; ++r) {
         const int64_t kv = kv_lens[r];
         const int32_t ql = q_lens ? q_lens[r] : 1;
@@ -61,10 +94,21 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
             }
         }
     }
+    if (units.overflow) return -2;
     const int32_t U = static_cast<int32_t>(units.size());
+    int64_t *start = buf.start;
+    int32_t *cta_begin = buf.cta_begin;
+    struct ItemList {
+        xllm_work_item *p;
+        int32_t n, cap;
+        bool overflow;
+        void push_back(const xllm_work_item &it) {
+            if (n < cap) p[n++] = it; else overflow = true;
+        }
+        size_t size() const { return (size_t)n; }
+    } items{buf.items, 0, buf.cap_items, false};
     // cost axis: start position of every unit.  A full tile costs tile_cost; the last tile of a unit is fetched
     // in 16-token steps: half of its cost is fixed, half goes with the volume; a unit's fixed cost grows with its row count.
-    std::vector<int64_t> start(static_cast<size_t>(U) + 1);
     start[0] = 0;
     for (int32_t u = 0; u < U; ++u) {
         Unit &un = units[u];
@@ -77,12 +121,11 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
     // Walk the axis once, CTA by CTA.  Each CTA aims at an equal share of what is still to be done; "what is
     // still to be done" includes the fixed cost a unit's continuation pays again when a cut splits the unit, so the
     // shares stay equal although every split adds work.
-    items.clear();
-    cta_begin.assign(static_cast<size_t>(n_ctas) + 1, 0);
+    for (int32_t c = 0; c <= n_ctas; ++c) cta_begin[c] = 0;
     int32_t n_partials = 0;
     int32_t u = 0, tile = 0;  // next work: unit u from tile `tile` on
     int64_t mean_overhead = 0;
-    for (const Unit &un : units) mean_overhead += un.overhead;
+    for (int32_t i = 0; i < U; ++i) mean_overhead += units[i].overhead;
     mean_overhead = U ? mean_overhead / U : 0;
     auto tiles_cost = [&](const Unit &un, int32_t from, int32_t to) -> int64_t {  // cost of tiles [from, to)
         if (to <= from) return 0;
@@ -140,6 +183,8 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
         }
     }
     cta_begin[n_ctas] = static_cast<int32_t>(items.size());
+    if (items.overflow) return -2;
+    if (n_items_out) *n_items_out = items.n;
     if (n_units_out) *n_units_out = U;
     if (n_partials_out) *n_partials_out = n_partials;
     return 0;

@@ -18,6 +18,28 @@ struct PlanTuning {
     int32_t min_piece_tiles = 6;  // pieces of a split unit are at least this many tiles (swept on B200: 4..8 are within noise)
 };
 
+struct PlanUnit {  // one (request, KV head, row group) on the planner's cost axis
+    int32_t req, kv_head;
+    int16_t q_tok0, n_q_tok, g0, n_g;
+    int32_t n_tiles;    // tiles that hold keys visible to the unit's last row
+    int32_t max_cut;    // largest tile boundary at which a split may start so that the first row still sees a key
+    int32_t last_cost;  // cost of the last (possibly short) tile
+    int32_t overhead;   // fixed cost of the unit: query load, hand-off to the epilogue, output rows
+};
+
+struct PlanBuffers {  // caller-provided work arrays of plan_partition_core
+    PlanUnit *units;
+    int64_t *start;     // cap_units + 1 entries
+    int32_t cap_units;
+    xllm_work_item *items;
+    int32_t cap_items;
+    int32_t *cta_begin;  // n_ctas + 1 entries
+};
+
+int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads);
+int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads,
+                        int32_t n_ctas, const PlanTuning &tune, const PlanBuffers &buf, int32_t *n_items_out,
+                        int32_t *n_units_out, int32_t *n_partials_out);
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
                    std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out);

@@ -204,6 +204,41 @@ xllm_status xllm_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *s
 xllm_status xllm_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
                                   const void *q, void *out, float *lse_out, float scale, void *cuda_stream);
 
+/* ---- decode attention without a context and without any allocation ------------------------------------------- */
+
+#define XLLM_STATIC_MAX_REQUESTS 64 /* requests per call of xllm_decode_attention_static */
+#define XLLM_STATIC_MAX_UNITS 512   /* requests x KV heads (x ceil(G / 16) when a GQA group has more than 16 heads) */
+
+/* (The paper has no counterpart of this entry point; it exists for a deployment constraint.)
+ *
+ * For callers that cannot allocate device memory where they call from -- an engine that gave all of its HBM to its
+ * own pools at start-up, a plugin living inside another runtime's memory budget, a path that must not run into
+ * cudaMalloc's implicit synchronisation -- and therefore cannot create an xllm_ctx (xllm_init allocates staging
+ * buffers, a partial-result workspace and events).  This call takes no context and calls no cudaMalloc, cudaFree,
+ * cudaHostAlloc or any other allocating routine, on the device or on the host: the split-KV kernel's work list, the
+ * fp32 partial results of split sequences, their arrival counters and a status word live in one fixed __device__
+ * array inside the library (about 2.7 MB, held by every GPU that loads the library until the process exits), and the
+ * host side plans in fixed static arrays.
+ *
+ * It computes what xllm_decode_attention computes (one query token per request) with the same kernels.
+ *   kv_ranges  host [n_req]: device address of each request's KV range, in the library's slot layout, i.e. filled by
+ *              xllm_kv_append (xllm_kv_slot_info().base of a slot) or a byte copy of such a range;
+ *   kv_lens    host [n_req]: tokens cached in each range (>= 1); the caller guarantees the ranges hold them;
+ *   q, out     device bf16 [n_req, H_q, D], 16-byte aligned;  lse_out device fp32 [n_req, H_q] or NULL.
+ * Limits: n_req <= XLLM_STATIC_MAX_REQUESTS and n_req * H_kv * ceil(G / 16) <= XLLM_STATIC_MAX_UNITS, head_dim 64 or
+ * 128; larger batches are refused with XLLM_ERR_UNSUPPORTED and a message (xllm_last_error(NULL)) before anything runs.
+ *
+ * The first call on a device does a one-time set-up with that device current: it looks up the array's device address
+ * (cudaGetSymbolAddress), clears the array and sets the kernels' shared-memory attribute.  Make that first call before
+ * any stream capture.  Every call first waits for the work already queued on `cuda_stream` (the previous call on that
+ * stream may still be using the array) and reads back the status word: if the previous call's kernel gave up a bounded
+ * wait, this call returns XLLM_ERR_CUDA (after launching its own work normally).  All calls share the one array, which
+ * keeps the last call's contents; what must start at zero is cleared by the call itself.  Calls whose kernels overlap
+ * on the GPU -- two streams, two threads -- race on it: serialise them.  Not re-entrant on the host either. */
+xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_t *kv_ranges, const int64_t *kv_lens, int32_t n_q_heads,
+                                         int32_t n_kv_heads, int32_t head_dim, const void *q, void *out, float *lse_out,
+                                         float scale, void *cuda_stream);
+
 /* ---- work partition (host only; exposed so that it can be checked without a GPU) ---------------------------- */
 
 /* Split the step's KV tile blocks into per-CTA runs of near-equal cost (hierarchical DP load balance,

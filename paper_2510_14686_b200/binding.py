@@ -93,6 +93,8 @@ EXPORTS = {
     "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
     "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_decode_attention_static": (ctypes.c_int32, [ctypes.c_int32, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                                       _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.POINTER(WorkItem), ctypes.c_int32, _i32p, _i32p, _i32p, _i32p]),
     "xllm_get_stats": (ctypes.c_int32, [_ctxp, ctypes.POINTER(Stats)]),
@@ -149,6 +151,24 @@ def plan_partition(kv_lens: Sequence[int], q_lens: Optional[Sequence[int]], n_q_
     if st != OK:
         raise XllmError(st, "xllm_plan_partition rejected the sizes")
     return [items[i] for i in range(n_items.value)], cta, n_units.value, n_parts.value
+
+
+STATIC_MAX_REQUESTS, STATIC_MAX_UNITS = 64, 512
+
+
+def decode_attention_static(kv_ranges, kv_lens, n_q_heads: int, n_kv_heads: int, head_dim: int, q, out, lse_out=None,
+                            scale: float = 1.0, stream=None):
+    """Context-free decode attention that allocates nothing (``xllm_decode_attention_static``).
+
+    For callers that may not allocate device memory: the kernel's scratch lives in a fixed array inside the library.
+    ``kv_ranges`` are device addresses of KV ranges in the library's slot layout, ``kv_lens`` their token counts.
+    """
+    r = np.ascontiguousarray(kv_ranges, dtype=np.uint64)
+    n = _i64(kv_lens)
+    st = _lib.xllm_decode_attention_static(len(r), r.ctypes.data, n.ctypes.data, n_q_heads, n_kv_heads, head_dim, _ptr(q),
+                                           _ptr(out), _ptr(lse_out), scale, _stream(stream))
+    if st != OK:
+        raise XllmError(st, _lib.xllm_last_error(None).decode())
 
 
 class Context:

@@ -31,6 +31,11 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+namespace xllm {
+// message returned by xllm_last_error(NULL): failures of calls that have no context
+void set_init_error(const char *msg) { g_init_error = msg ? msg : ""; }
+}  // namespace xllm
+
 struct xllm_ctx {
     xllm_config cfg{};
     std::unique_ptr<XTensor> xt;

@@ -1,0 +1,237 @@
+// xllm_decode_attention_static: decode attention for callers that may not allocate.
+//
+// Some hosts of this library run where no device allocation can be made while they are serving: an engine that
+// has handed all of its HBM to its own pools at start-up, a plugin that runs inside another runtime's memory budget,
+// code that sits on a path where cudaMalloc's implicit device synchronisation is not acceptable.  The normal
+// entry points need an xllm_ctx, and creating one allocates (staging buffers, partial-result workspace, events).
+// This entry point needs no context: everything the split-KV attention kernel needs beyond its inputs and outputs
+// -- the work list, the fp32 partial results of split sequences, their arrival counters, a status word -- lives in one
+// file-scope __device__ array of fixed size that every GPU loading the library carries until the process exits.
+// The price is a modest upper bound on the batch (see the limits below), no verification (q_len = 1 only), and no
+// concurrency: every call shares the one array.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "xllm_attn.h"
+#include "xllm_internal.h"
+
+namespace xllm {
+void set_init_error(const char *msg);  // api.cpp: text returned by xllm_last_error(NULL)
+}
+
+using namespace xllm;
+
+namespace {
+
+constexpr int kMaxRequests = XLLM_STATIC_MAX_REQUESTS;
+constexpr int kMaxUnits = XLLM_STATIC_MAX_UNITS;
+constexpr int kMaxItems = kMaxUnits + kMaxCtas;
+constexpr int kMaxPartials = 2 * kMaxCtas + 2;
+constexpr int kMaxDevices = 64;
+
+struct Scratch {
+    DevItem items[kMaxItems];
+    CombineDesc combine[kMaxPartials];
+    float part_o[(size_t)kMaxPartials * kMaxRows * 128];
+    float part_lse[(size_t)kMaxPartials * kMaxRows];
+    int32_t counters[kMaxPartials];  // must be zero when a launch starts
+    int32_t error;                   // set by a kernel whose bounded wait expired; read back by the next call
+};
+
+// The scratch memory itself (about 2.7 MB per GPU).  In host code this name is only a handle for the runtime: its
+// device address is obtained once per device with cudaGetSymbolAddress and passed to the kernels as a pointer.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(Scratch)];
+
+struct DeviceState {
+    Scratch *scratch = nullptr;  // device address of g_static_scratch on that device
+    int sm_count = 0;
+    bool configured[2] = {false, false};  // kernel attributes set for head_dim 64 / 128
+};
+DeviceState g_dev[kMaxDevices];
+
+// Host-side work arrays of fixed capacity (the call is not re-entrant).
+PlanUnit g_units[kMaxUnits];
+int64_t g_start[kMaxUnits + 1];
+xllm_work_item g_items[kMaxItems];
+int32_t g_cta_begin[kMaxCtas + 1];
+DevItem g_dev_items[kMaxItems];
+CombineDesc g_combine[kMaxPartials];
+int32_t g_part_first[kMaxPartials], g_part_count[kMaxPartials];
+
+xllm_status fail(xllm_status code, const char *msg) {
+    set_init_error(msg);
+    return code;
+}
+
+}  // namespace
+
+extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_t *kv_ranges, const int64_t *kv_lens,
+                                                    int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, const void *q,
+                                                    void *out, float *lse_out, float scale, void *cuda_stream) {
+    char msg[256];
+    if (n_req < 1 || !kv_ranges || !kv_lens || !q || !out)
+        return fail(XLLM_ERR_INVALID, "decode_attention_static: n_req must be >= 1 and the pointers non-null");
+    if (n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads)
+        return fail(XLLM_ERR_INVALID, "decode_attention_static: n_q_heads must be a positive multiple of n_kv_heads");
+    if (head_dim != 64 && head_dim != 128) return fail(XLLM_ERR_UNSUPPORTED, "decode_attention_static: head_dim must be 64 or 128");
+    if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return fail(XLLM_ERR_INVALID, "decode_attention_static: q and out must be 16-byte aligned");
+    if (!(scale > 0.f) || !std::isfinite(scale)) return fail(XLLM_ERR_INVALID, "decode_attention_static: scale must be finite and > 0");
+    const int64_t n_units = plan_count_units(n_req, nullptr, n_q_heads, n_kv_heads);
+    if (n_req > kMaxRequests || n_units > kMaxUnits) {
+        std::snprintf(msg, sizeof msg,
+                      "decode_attention_static: batch too large for the static scratch array: %d requests (max %d), %lld "
+                      "(request, KV head, row group) units (max %d); use xllm_decode_attention with a context instead",
+                      n_req, kMaxRequests, (long long)n_units, kMaxUnits);
+        return fail(XLLM_ERR_UNSUPPORTED, msg);
+    }
+    for (int32_t i = 0; i < n_req; ++i) {
+        if (kv_lens[i] < 1 || kv_lens[i] > (int64_t)INT32_MAX - XLLM_TILE_TOKENS)
+            return fail(XLLM_ERR_INVALID, "decode_attention_static: every kv_len must be >= 1 (and below 2^31)");
+        if (kv_ranges[i] == 0 || (kv_ranges[i] & 15)) return fail(XLLM_ERR_INVALID, "decode_attention_static: bad KV range address");
+    }
+
+    // ---- set-up, once per device, with that device current ----
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) return fail(XLLM_ERR_CUDA, "decode_attention_static: no current CUDA device");
+    DeviceState &ds = g_dev[dev];
+    if (!ds.scratch) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) {
+            std::snprintf(msg, sizeof msg, "decode_attention_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            return fail(XLLM_ERR_CUDA, msg);
+        }
+        int major = 0, sms = 0;
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (major != 10) return fail(XLLM_ERR_UNSUPPORTED, "decode_attention_static: kernels are built for sm_100a only");
+        e = cudaMemset(ptr, 0, sizeof(Scratch));  // counters and status word start at zero
+        if (e != cudaSuccess) return fail(XLLM_ERR_CUDA, "decode_attention_static: clearing the scratch array failed");
+        ds.sm_count = sms < kMaxCtas ? sms : kMaxCtas;
+        ds.scratch = static_cast<Scratch *>(ptr);
+    }
+    if (!ds.configured[head_dim == 128]) {
+        e = (cudaError_t)configure_kernels(head_dim);
+        if (e != cudaSuccess) return fail(XLLM_ERR_CUDA, "decode_attention_static: cudaFuncSetAttribute failed");
+        ds.configured[head_dim == 128] = true;
+    }
+    Scratch *sc = ds.scratch;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    // ---- wait for what is queued on the stream (the previous call on it still owns the scratch array) and read
+    //      the status word it may have left ----
+    int32_t status = 0;
+    e = cudaMemcpyAsync(&status, &sc->error, sizeof status, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) {
+        std::snprintf(msg, sizeof msg, "decode_attention_static: %s", cudaGetErrorString(e));
+        return fail(XLLM_ERR_CUDA, msg);
+    }
+    bool stale = status != 0;
+
+    // ---- plan the work in the fixed host arrays ----
+    PlanTuning tune;
+    PlanBuffers buf{g_units, g_start, kMaxUnits, g_items, kMaxItems, g_cta_begin};
+    int32_t n_items = 0, n_units_planned = 0, n_partials = 0;
+    if (plan_partition_core(n_req, kv_lens, nullptr, n_q_heads, n_kv_heads, ds.sm_count, tune, buf, &n_items, &n_units_planned,
+                            &n_partials) != 0 || n_partials > kMaxPartials)
+        return fail(XLLM_ERR_UNSUPPORTED, "decode_attention_static: the work list does not fit the static arrays");
+    const int32_t G = n_q_heads / n_kv_heads;
+    const int64_t head_tile = head_tile_bytes(head_dim);
+    int32_t n_combine = 0;
+    {
+        int32_t last_unit = -1, first = 0;
+        for (int32_t i = 0; i < n_partials; ++i) g_part_count[i] = 0;
+        for (int32_t i = 0; i < n_items; ++i) {
+            const xllm_work_item &it = g_items[i];
+            if (it.partial_idx < 0) continue;
+            if (it.unit != last_unit) {
+                last_unit = it.unit;
+                first = it.partial_idx;
+            }
+            g_part_first[it.partial_idx] = first;
+            ++g_part_count[first];
+        }
+        for (int32_t i = 0; i < n_items; ++i) {
+            const xllm_work_item &it = g_items[i];
+            if (it.partial_idx < 0 || g_part_first[it.partial_idx] != it.partial_idx) continue;
+            if (g_part_count[it.partial_idx] > kFuseMaxParts)
+                g_combine[n_combine++] = {it.partial_idx, g_part_count[it.partial_idx], it.req + it.q_tok0, it.kv_head * G + it.g0,
+                                          it.n_q_tok, it.n_g};
+        }
+    }
+    for (int32_t i = 0; i < n_items; ++i) {
+        const xllm_work_item &w = g_items[i];
+        DevItem &d = g_dev_items[i];
+        d.kv = kv_ranges[w.req] + (uint64_t)(w.kv_head * head_tile);
+        d.q_row = w.req + w.q_tok0;  // q_len = 1: request r owns row r
+        d.partial_idx = w.partial_idx;
+        d.tile_begin = w.tile_begin;
+        d.tile_end = w.tile_end;
+        d.kv_end = (int32_t)kv_lens[w.req] - 1 + w.q_tok0 + w.n_q_tok;
+        d.head0 = (int16_t)(w.kv_head * G + w.g0);
+        d.n_q_tok = (uint8_t)w.n_q_tok;
+        d.n_g = (uint8_t)w.n_g;
+        d.part_first = w.partial_idx >= 0 ? g_part_first[w.partial_idx] : 0;
+        const int32_t pieces = w.partial_idx >= 0 ? g_part_count[d.part_first] : 0;
+        d.n_parts = pieces <= kFuseMaxParts ? pieces : 0;
+        d.pad[0] = d.pad[1] = 0;
+    }
+
+    // ---- stage the lists in the scratch array (copies from pageable memory are staged by the driver before the
+    //      call returns, so the host arrays may be reused at once), clear what must start at zero, launch ----
+    e = cudaMemcpyAsync(sc->items, g_dev_items, sizeof(DevItem) * (size_t)n_items, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && n_combine)
+        e = cudaMemcpyAsync(sc->combine, g_combine, sizeof(CombineDesc) * (size_t)n_combine, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && stale) e = cudaMemsetAsync(sc->counters, 0, sizeof sc->counters, stream);  // an aborted launch left them behind
+    if (e == cudaSuccess && stale) e = cudaMemsetAsync(&sc->error, 0, sizeof sc->error, stream);
+    if (e != cudaSuccess) {
+        std::snprintf(msg, sizeof msg, "decode_attention_static: staging the work list: %s", cudaGetErrorString(e));
+        return fail(XLLM_ERR_CUDA, msg);
+    }
+    AttnLaunch al{};
+    al.items = sc->items;
+    al.q = q;
+    al.out = out;
+    al.lse_out = lse_out;
+    al.part_o = sc->part_o;
+    al.part_lse = sc->part_lse;
+    al.counters = sc->counters;
+    al.error_flag = &sc->error;
+    al.trace = nullptr;
+    al.n_q_heads = n_q_heads;
+    al.n_kv_heads = n_kv_heads;
+    al.head_dim = head_dim;
+    al.scale_log2 = scale * 1.4426950408889634f;
+    al.n_ctas = ds.sm_count;
+    std::memcpy(al.cta_begin, g_cta_begin, sizeof(int32_t) * (size_t)(ds.sm_count + 1));
+    for (int32_t c = 0; c < ds.sm_count; ++c)
+        if (al.cta_begin[c] < al.cta_begin[c + 1]) al.first_item[c] = g_dev_items[al.cta_begin[c]];
+    int le = launch_attention(al, stream);
+    if (le == 0 && n_combine) {
+        CombineLaunch cl{};
+        cl.descs = sc->combine;
+        cl.n_units = n_combine;
+        cl.part_o = sc->part_o;
+        cl.part_lse = sc->part_lse;
+        cl.out = out;
+        cl.lse_out = lse_out;
+        cl.n_q_heads = n_q_heads;
+        cl.head_dim = head_dim;
+        le = launch_combine(cl, stream);
+    }
+    if (le != 0) {
+        std::snprintf(msg, sizeof msg, "decode_attention_static: kernel launch failed: %s", cudaGetErrorString((cudaError_t)le));
+        return fail(XLLM_ERR_CUDA, msg);
+    }
+    if (stale)
+        return fail(XLLM_ERR_CUDA,
+                    "decode_attention_static: the PREVIOUS call's kernel gave up a bounded wait, its output is invalid "
+                    "(this call was launched normally)");
+    return XLLM_OK;
+}

@@ -1,0 +1,91 @@
+"""GPU: the context-free, allocation-free decode entry point against the normal one.
+
+Who needs it: callers that cannot allocate device memory where they call from (an engine that handed all of its
+HBM to its own pools at start-up, a plugin inside another runtime's memory budget) and so cannot create a library
+context.  ``xllm_decode_attention_static`` keeps the kernel's scratch (work list, partial results of split
+sequences, arrival counters, status word) in one fixed array inside the library.  Here the KV ranges are filled
+through a normal context, then the same ranges are handed to the static entry point by address, twice in a row (the
+second call re-uses the array the first one left behind), and both results must equal the normal entry point's.
+
+This file is collected last on purpose, and passes both alone in a fresh process and after the other tests.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_14686_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+def _run(binding, batch):
+    import gpu_harness as gh
+
+    s = batch.shape
+    lens = [r.kv_len for r in batch.requests]
+    with gh.make_ctx(binding, s, len(lens), max(lens) + 8, lens) as ctx:
+        slots = gh.load_requests(ctx, batch.requests)
+        ref_bits, ref_lse = gh.run_attention(ctx, batch, slots)              # existing entry point
+        st = ctx.get_stats()
+        ranges = np.array([ctx.kv_slot_info(sl).base for sl in slots], np.uint64)
+        kv_lens = np.array(lens, np.int64)
+        q = gh.dev_bits(np.concatenate([r.q for r in batch.requests], axis=0))
+        results = []
+        for call in range(2):                                                # two calls in a row share the scratch array
+            out = torch.zeros((len(lens), s.n_q_heads, s.head_dim), dtype=torch.int16, device="cuda")
+            lse = torch.full((len(lens), s.n_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+            binding.decode_attention_static(ranges, kv_lens, s.n_q_heads, s.n_kv_heads, s.head_dim, q, out, lse, s.scale)
+            torch.cuda.synchronize()
+            results.append((gh.host_bits(out), lse.cpu().numpy()))
+    return ref_bits, ref_lse, results, st
+
+
+@pytest.mark.parametrize("hq,hkv,d,lens", [
+    (8, 2, 64, [273, 190, 249, 21, 1, 64, 65]),                  # small, nothing split
+    (28, 4, 128, [3000, 517, 4060, 1931, 64, 2200]),             # split units merged inside the attention kernel
+    (8, 1, 128, [50000, 300]),                                   # one sequence in > 8 pieces: combine kernel path
+])
+def test_static_entry_matches_context_entry_twice(binding, hq, hkv, d, lens):
+    import gpu_harness as gh
+
+    batch = wl.custom_batch(900 + hq + d, hq, hkv, d, lens)
+    ref_bits, ref_lse, results, st = _run(binding, batch)
+    if max(lens) >= 3000:
+        assert st.partial_items > 0                                   # the scratch array really was used
+    ref = wl.bits_to_f64(ref_bits)
+    for out_bits, lse in results:
+        got = wl.bits_to_f64(out_bits)
+        assert np.isfinite(got).all()
+        err = np.abs(got - ref)
+        assert err.max() <= gh.MAX_ABS and err.mean() <= gh.MEAN_ABS  # the tolerance of the parity tests
+        assert np.abs(lse - ref_lse).max() <= gh.LSE_ABS
+    # and against the oracle, like every other parity case
+    gh.assert_parity(results[1][0], results[1][1], *gh.oracle_batch(batch)) if max(lens) >= 500 else None
+
+
+def test_static_entry_refuses_oversized_batches_with_a_clear_error(binding):
+    q = torch.zeros((80, 8, 64), dtype=torch.int16, device="cuda")
+    out = torch.zeros_like(q)
+    ranges = np.full(80, q.data_ptr(), np.uint64)
+    with pytest.raises(binding.XllmError) as e:                       # 80 requests > 64
+        binding.decode_attention_static(ranges, np.full(80, 10, np.int64), 8, 2, 64, q, out, None, 0.125)
+    assert e.value.status == binding.ERR_UNSUPPORTED and "max 64" in str(e.value)
+    with pytest.raises(binding.XllmError) as e:                       # 40 requests x 16 KV heads = 640 units > 512
+        binding.decode_attention_static(ranges[:40], np.full(40, 10, np.int64), 16, 16, 64, q, out, None, 0.125)
+    assert e.value.status == binding.ERR_UNSUPPORTED and "max 512" in str(e.value)
+    for bad in (lambda: binding.decode_attention_static(ranges[:2], np.array([10, 0], np.int64), 8, 2, 64, q, out, None, 0.125),
+                lambda: binding.decode_attention_static(ranges[:2], np.array([10, 10], np.int64), 8, 3, 64, q, out, None, 0.125),
+                lambda: binding.decode_attention_static(ranges[:2], np.array([10, 10], np.int64), 8, 2, 64, q, out, None, -1.0)):
+        with pytest.raises(binding.XllmError) as e:
+            bad()
+        assert e.value.status == binding.ERR_INVALID
+    with pytest.raises(binding.XllmError) as e:
+        binding.decode_attention_static(ranges[:2], np.array([10, 10], np.int64), 8, 2, 96, q, out, None, 0.125)
+    assert e.value.status == binding.ERR_UNSUPPORTED

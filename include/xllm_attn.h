@@ -108,6 +108,8 @@ typedef struct {
     int32_t partial_idx; /* -1: the item covers the whole context and writes the final output;
                             else index of its partial result in the split workspace */
     int32_t unit;        /* id of the (request, KV head, row group) unit the item belongs to */
+    int32_t part_first;  /* partial_idx of the unit's first piece (pieces of a unit have consecutive indices); 0 if whole */
+    int32_t n_parts;     /* number of pieces the unit was cut into; 0 if whole */
 } xllm_work_item;
 
 /* ---- life cycle ------------------------------------------------------------------------------- */

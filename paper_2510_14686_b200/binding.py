@@ -67,7 +67,8 @@ class SlotInfo(ctypes.Structure):
 class WorkItem(ctypes.Structure):
     _fields_ = [("req", ctypes.c_int32), ("kv_head", ctypes.c_int32), ("tile_begin", ctypes.c_int32),
                 ("tile_end", ctypes.c_int32), ("q_tok0", ctypes.c_int16), ("n_q_tok", ctypes.c_int16),
-                ("g0", ctypes.c_int16), ("n_g", ctypes.c_int16), ("partial_idx", ctypes.c_int32), ("unit", ctypes.c_int32)]
+                ("g0", ctypes.c_int16), ("n_g", ctypes.c_int16), ("partial_idx", ctypes.c_int32), ("unit", ctypes.c_int32),
+                ("part_first", ctypes.c_int32), ("n_parts", ctypes.c_int32)]
 
 
 _vp, _i32p, _i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)

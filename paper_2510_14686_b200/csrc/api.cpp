@@ -69,7 +69,7 @@ struct xllm_ctx {
     xllm_stats st{};
 
     std::vector<xllm_work_item> items;
-    std::vector<int32_t> cta_begin, q_row0, part_first, part_count;
+    std::vector<int32_t> cta_begin, q_row0;
     std::vector<CombineDesc> combine;
     std::vector<int64_t> kv_lens;
     std::vector<uint8_t> seen;
@@ -228,29 +228,12 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
             acc += q_lens ? q_lens[i] : 1;
         }
     }
-    std::vector<int32_t> &part_first = ctx->part_first, &part_count = ctx->part_count;  // indexed by partial slot
-    part_first.assign((size_t)n_partials, 0);
-    part_count.assign((size_t)n_partials, 0);
     std::vector<CombineDesc> &combine = ctx->combine;
     combine.clear();
-    {
-        int32_t last_unit = -1, first = 0;
-        for (const xllm_work_item &it : ctx->items) {
-            if (it.partial_idx < 0) continue;
-            if (it.unit != last_unit) {
-                last_unit = it.unit;
-                first = it.partial_idx;
-            }
-            part_first[(size_t)it.partial_idx] = first;
-            ++part_count[(size_t)first];
-        }
-        for (const xllm_work_item &it : ctx->items) {
-            if (it.partial_idx < 0 || part_first[(size_t)it.partial_idx] != it.partial_idx) continue;  // first piece only
-            if (part_count[(size_t)it.partial_idx] > kFuseMaxParts)
-                combine.push_back({it.partial_idx, part_count[(size_t)it.partial_idx], q_row0[(size_t)it.req] + it.q_tok0,
-                                   it.kv_head * G + it.g0, it.n_q_tok, it.n_g});
-        }
-    }
+    for (const xllm_work_item &it : ctx->items)
+        if (it.partial_idx >= 0 && it.partial_idx == it.part_first && it.n_parts > kFuseMaxParts)  // first piece of a unit
+            combine.push_back({it.part_first, it.n_parts, q_row0[(size_t)it.req] + it.q_tok0, it.kv_head * G + it.g0, it.n_q_tok,
+                               it.n_g});
 
     int idx;
     int e = acquire_stage(ctx, &idx);
@@ -276,9 +259,8 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         di[i].head0 = (int16_t)(w.kv_head * G + w.g0);
         di[i].n_q_tok = (uint8_t)w.n_q_tok;
         di[i].n_g = (uint8_t)w.n_g;
-        di[i].part_first = w.partial_idx >= 0 ? part_first[(size_t)w.partial_idx] : 0;
-        const int32_t pieces = w.partial_idx >= 0 ? part_count[(size_t)di[i].part_first] : 0;
-        di[i].n_parts = pieces <= kFuseMaxParts ? pieces : 0;
+        di[i].part_first = w.part_first;
+        di[i].n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
         di[i].pad[0] = di[i].pad[1] = 0;
     }
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
@@ -380,13 +362,14 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         drv = make_cuda_driver(&derr);
         if (!drv) return bad(XLLM_ERR_CUDA, derr);
     }
-    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece": planner cost model override (tuning aid)
-        int a, b, c, d;
-        if (std::sscanf(t, "%d,%d,%d,%d", &a, &b, &c, &d) == 4 && a > 0 && b >= 0 && c >= 0 && d >= 1) {
+    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece[,pieces_first]": planner override (tuning aid)
+        int a, b, c, d, f = 1;
+        if (std::sscanf(t, "%d,%d,%d,%d,%d", &a, &b, &c, &d, &f) >= 4 && a > 0 && b >= 0 && c >= 0 && d >= 1) {
             ctx->tune.tile_cost = a;
             ctx->tune.unit_overhead = b;
             ctx->tune.row_overhead = c;
             ctx->tune.min_piece_tiles = d;
+            ctx->tune.pieces_first = f;
         }
     }
     ctx->xt.reset(new XTensor(std::move(drv), cfg->device, cfg->max_slots, cfg->max_seq_len, row_bytes));

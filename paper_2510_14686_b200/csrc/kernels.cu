@@ -354,6 +354,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     __syncthreads();          // barriers initialised
     grid_launch_dependents();  // the next kernel of the stream may start its own prologue
     grid_dependency_wait();    // from here on q, the KV ranges and the outputs may be touched
+    const unsigned long long g_go = TRACE ? globaltimer_ns() : 0ull;
+    unsigned long long g_first = 0, g_last = 0;
 
     for (int batch_lo = item_lo; batch_lo < item_hi; batch_lo += kItemBatch) {
         const int nb = min(kItemBatch, item_hi - batch_lo);
@@ -486,7 +488,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                         if (mask) XLLM_TILE(true, false); else XLLM_TILE(false, false);
                     }
 #undef XLLM_TILE
-                    if (TRACE && !tr_first) tr_first = clock64() - t_start;
+                    if (TRACE && !tr_first) {
+                        tr_first = clock64() - t_start;
+                        g_first = globaltimer_ns();
+                    }
+                    if (TRACE) g_last = globaltimer_ns();
                 }
                 if (TRACE) {
                     const unsigned long long t1 = clock64();
@@ -613,15 +619,16 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         item_seq += nb;
     }
 
-    // trace layout (16 words per CTA): 0 cycles of warp 0, 1 cycles to its first finished tile, 2 cycles in tile loops
-    // (warp 0), 3 global-timer ns at CTA start (9: at the end of warp 4), 4 waiting for query rows, 5 item hand-off incl. waiting for the epilogue, 6 items, 7 tiles,
-    // 8/10 the same as 2/5 for warp 4, 11 producer cycles waiting for free ring slots, 12 producer cycles,
-    // 13 epilogue busy cycles, 14 epilogue cycles, 15 nanoseconds of warp 0 (global timer).
+    // trace layout (16 words per CTA); "ns" = absolute global-timer nanoseconds, "cycles" = SM clock cycles.
+    // Warp 0: 0 ns after the dependency wait, 1 ns at its first finished tile, 2 ns at its last finished tile, 3 ns at
+    // CTA start, 4 cycles waiting for query rows, 5 cycles in item hand-off (incl. waiting for the epilogue), 6 items,
+    // 7 tiles, 15 ns lifetime.  Warp 4: 8 cycles in tile loops, 9 ns at its end, 10 cycles in hand-off.  Producer: 11
+    // cycles waiting for free ring slots, 12 cycles lifetime.  Epilogue warp 9: 13 busy cycles, 14 ns at its end.
     if (TRACE && lane == 0 && (warp == 0 || warp == 4 || warp == kProducerWarp || warp == kEpilogueWarp0)) {
         unsigned long long *tr = p.trace + (int64_t)blockIdx.x * kTraceWords;
         const unsigned long long total = clock64() - t_start;
         if (warp == 0) {
-            tr[0] = total; tr[1] = tr_first; tr[2] = tr_tiles; tr[3] = g_start; tr[4] = tr_wait_q; tr[5] = tr_switch;
+            tr[0] = g_go; tr[1] = g_first; tr[2] = g_last; tr[3] = g_start; tr[4] = tr_wait_q; tr[5] = tr_switch;
             tr[6] = (unsigned long long)(item_hi - item_lo); tr[7] = fill;
             tr[15] = globaltimer_ns() - g_start;
         } else if (warp == 4) {
@@ -629,7 +636,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         } else if (warp == kProducerWarp) {
             tr[11] = tr_wait_empty; tr[12] = total;
         } else {
-            tr[13] = tr_epi; tr[14] = total;
+            tr[13] = tr_epi; tr[14] = globaltimer_ns();
         }
     }
 

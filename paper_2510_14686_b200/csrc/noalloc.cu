@@ -59,7 +59,6 @@ xllm_work_item g_items[kMaxItems];
 int32_t g_cta_begin[kMaxCtas + 1];
 DevItem g_dev_items[kMaxItems];
 CombineDesc g_combine[kMaxPartials];
-int32_t g_part_first[kMaxPartials], g_part_count[kMaxPartials];
 
 xllm_status fail(xllm_status code, const char *msg) {
     set_init_error(msg);
@@ -144,26 +143,10 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
     const int32_t G = n_q_heads / n_kv_heads;
     const int64_t head_tile = head_tile_bytes(head_dim);
     int32_t n_combine = 0;
-    {
-        int32_t last_unit = -1, first = 0;
-        for (int32_t i = 0; i < n_partials; ++i) g_part_count[i] = 0;
-        for (int32_t i = 0; i < n_items; ++i) {
-            const xllm_work_item &it = g_items[i];
-            if (it.partial_idx < 0) continue;
-            if (it.unit != last_unit) {
-                last_unit = it.unit;
-                first = it.partial_idx;
-            }
-            g_part_first[it.partial_idx] = first;
-            ++g_part_count[first];
-        }
-        for (int32_t i = 0; i < n_items; ++i) {
-            const xllm_work_item &it = g_items[i];
-            if (it.partial_idx < 0 || g_part_first[it.partial_idx] != it.partial_idx) continue;
-            if (g_part_count[it.partial_idx] > kFuseMaxParts)
-                g_combine[n_combine++] = {it.partial_idx, g_part_count[it.partial_idx], it.req + it.q_tok0, it.kv_head * G + it.g0,
-                                          it.n_q_tok, it.n_g};
-        }
+    for (int32_t i = 0; i < n_items; ++i) {
+        const xllm_work_item &it = g_items[i];
+        if (it.partial_idx >= 0 && it.partial_idx == it.part_first && it.n_parts > kFuseMaxParts)  // first piece of a unit
+            g_combine[n_combine++] = {it.part_first, it.n_parts, it.req + it.q_tok0, it.kv_head * G + it.g0, it.n_q_tok, it.n_g};
     }
     for (int32_t i = 0; i < n_items; ++i) {
         const xllm_work_item &w = g_items[i];
@@ -177,9 +160,8 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
         d.head0 = (int16_t)(w.kv_head * G + w.g0);
         d.n_q_tok = (uint8_t)w.n_q_tok;
         d.n_g = (uint8_t)w.n_g;
-        d.part_first = w.partial_idx >= 0 ? g_part_first[w.partial_idx] : 0;
-        const int32_t pieces = w.partial_idx >= 0 ? g_part_count[d.part_first] : 0;
-        d.n_parts = pieces <= kFuseMaxParts ? pieces : 0;
+        d.part_first = w.part_first;
+        d.n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
         d.pad[0] = d.pad[1] = 0;
     }
 

@@ -171,6 +171,8 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
             it.n_g = un.n_g;
             it.partial_idx = (tile == 0 && take == un.n_tiles) ? -1 : n_partials++;
             it.unit = u;
+            it.part_first = 0;
+            it.n_parts = 0;
             items.push_back(it);
             load += un.overhead + tiles_cost(un, tile, tile + take);
             tile += take;
@@ -184,6 +186,32 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     }
     cta_begin[n_ctas] = static_cast<int32_t>(items.size());
     if (items.overflow) return -2;
+    // Pieces of one unit are adjacent in walk order: give each its unit's first slot and piece count ...
+    for (int32_t i = 0; i < items.n;) {
+        if (items.p[i].partial_idx < 0) {
+            ++i;
+            continue;
+        }
+        int32_t j = i;
+        while (j < items.n && items.p[j].unit == items.p[i].unit) ++j;
+        for (int32_t k = i; k < j; ++k) {
+            items.p[k].part_first = items.p[i].partial_idx;
+            items.p[k].n_parts = j - i;
+        }
+        i = j;
+    }
+    // ... then, optionally, let every CTA do its pieces first so that the round trip of their partial results through
+    // global memory is not at the very end of the CTA's run (off by default: it measured 2-4 % slower on B200).
+    // (in place and order preserving, by rotation: a CTA holds at most two pieces, and nothing is allocated)
+    for (int32_t c = 0; c < n_ctas && tune.pieces_first; ++c) {
+        int32_t front = cta_begin[c];
+        for (int32_t i = cta_begin[c]; i < cta_begin[c + 1]; ++i) {
+            if (items.p[i].partial_idx < 0) continue;
+            const xllm_work_item piece = items.p[i];
+            for (int32_t k = i; k > front; --k) items.p[k] = items.p[k - 1];
+            items.p[front++] = piece;
+        }
+    }
     if (n_items_out) *n_items_out = items.n;
     if (n_units_out) *n_units_out = U;
     if (n_partials_out) *n_partials_out = n_partials;

@@ -15,6 +15,7 @@ struct PlanTuning {
     int32_t tile_cost = 8;        // cost of one full KV tile block on the partition axis
     int32_t unit_overhead = 6;    // fixed cost of starting a unit (Q load, hand-off, output), same scale ...
     int32_t row_overhead = 8;     // ... plus this much for a full 16-row unit, in proportion to its rows
+    int32_t pieces_first = 0;     // 1: inside a CTA the pieces of split units run before the whole units (measured slower on B200)
     int32_t min_piece_tiles = 6;  // pieces of a split unit are at least this many tiles (swept on B200: 4..8 are within noise)
 };
 

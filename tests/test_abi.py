@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(binding):
 
 
 def test_struct_sizes_match_header_layout(binding):
-    assert ctypes.sizeof(binding.WorkItem) == 32
+    assert ctypes.sizeof(binding.WorkItem) == 40
     assert ctypes.sizeof(binding.Config) == 56
     assert ctypes.sizeof(binding.SlotInfo) == 48
 

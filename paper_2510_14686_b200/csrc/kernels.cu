@@ -575,40 +575,68 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 if (lane == 0) mbar_arrive(bar_mempty);  // the consumers may overwrite the group states
                 if (live && it.partial_idx >= 0 && it.n_parts > 0) {
                     // Lightly split unit: whichever piece finishes last merges all pieces (log-sum-exp) and writes the
-                    // final rows, so no second launch is needed.  Release: partial stores, fence, barrier, one atomic.
-                    // Acquire: atomic result, barrier, fence, loads that bypass L1.
+                    // final rows, so no second launch is needed.
+                    // Release: every epilogue thread's partial stores, CTA barrier, then ONE acq_rel atomic at GPU scope
+                    // by thread 0 (cumulative over what the barrier made visible to it).  Acquire: that atomic, CTA
+                    // barrier, loads that bypass L1.
                     volatile int *bcast = reinterpret_cast<volatile int *>(smem + C::kOffFlags) + 1;
-                    __threadfence();
                     asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");
-                    if (et == 0) *bcast = atomicAdd(p.counters + it.part_first, 1);
+                    if (et == 0) {
+                        int old;
+                        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.counters + it.part_first) : "memory");
+                        *bcast = old;
+                    }
                     asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");
                     if (*bcast == it.n_parts - 1) {
-                        __threadfence();
-                        for (int idx = et; idx < n_rows * kC4; idx += kEpilogueThreads) {
-                            const int row = idx / kC4, c4 = idx - row * kC4;
-                            float M = -INFINITY;
-                            for (int s2 = 0; s2 < it.n_parts; ++s2)
-                                M = fmaxf(M, __ldcg(p.part_lse + (int64_t)(it.part_first + s2) * kMaxRows + row));
-                            const float Ms = (M == -INFINITY) ? 0.f : M;
-                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                            float W = 0.f;
-                            for (int s2 = 0; s2 < it.n_parts; ++s2) {
-                                const int64_t pi = it.part_first + s2;
-                                const float w = exp2f(__ldcg(p.part_lse + pi * kMaxRows + row) - Ms);  // 0 for a piece without keys
-                                const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.part_o + (pi * kMaxRows + row) * D) + c4);
-                                W += w;
-                                acc.x += w * v.x;
-                                acc.y += w * v.y;
-                                acc.z += w * v.z;
-                                acc.w += w * v.w;
+                        // All loads of up to kIdx output elements are issued before any is used (the pieces sit in L2, a
+                        // round trip costs ~0.7 us under load); n_parts <= kFuseMaxParts, unrolled with predicates.
+                        constexpr int kIdx = 3;
+                        for (int base = et; base < n_rows * kC4; base += kIdx * kEpilogueThreads) {
+                            float ls[kIdx][kFuseMaxParts];
+                            float4 v[kIdx][kFuseMaxParts];
+#pragma unroll
+                            for (int j = 0; j < kIdx; ++j) {
+                                const int idx = base + j * kEpilogueThreads;
+                                const int row = idx / kC4, c4 = idx - row * kC4;
+#pragma unroll
+                                for (int s2 = 0; s2 < kFuseMaxParts; ++s2) {
+                                    const int64_t pi = it.part_first + s2;
+                                    ls[j][s2] = -INFINITY;  // weight 0 for the padding
+                                    v[j][s2] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    if (s2 < it.n_parts && idx < n_rows * kC4) {
+                                        ls[j][s2] = __ldcg(p.part_lse + pi * kMaxRows + row);
+                                        v[j][s2] = __ldcg(reinterpret_cast<const float4 *>(p.part_o + (pi * kMaxRows + row) * D) + c4);
+                                    }
+                                }
                             }
-                            const float inv = (W > 0.f) ? 1.f / W : 0.f;
-                            const int ti = row / it.n_g, gi = row - ti * it.n_g;
-                            const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
-                            *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
-                                make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-                            if (c4 == 0 && p.lse_out)
-                                p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
+#pragma unroll
+                            for (int j = 0; j < kIdx; ++j) {
+                                const int idx = base + j * kEpilogueThreads;
+                                if (idx >= n_rows * kC4) break;
+                                const int row = idx / kC4, c4 = idx - row * kC4;
+                                float M = -INFINITY;
+#pragma unroll
+                                for (int s2 = 0; s2 < kFuseMaxParts; ++s2) M = fmaxf(M, ls[j][s2]);
+                                const float Ms = (M == -INFINITY) ? 0.f : M;
+                                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                                float W = 0.f;
+#pragma unroll
+                                for (int s2 = 0; s2 < kFuseMaxParts; ++s2) {  // fixed order: repeatable bit for bit
+                                    const float w = exp2f(ls[j][s2] - Ms);     // 0 for a piece without keys and for padding
+                                    W += w;
+                                    acc.x += w * v[j][s2].x;
+                                    acc.y += w * v[j][s2].y;
+                                    acc.z += w * v[j][s2].z;
+                                    acc.w += w * v[j][s2].w;
+                                }
+                                const float inv = (W > 0.f) ? 1.f / W : 0.f;
+                                const int ti = row / it.n_g, gi = row - ti * it.n_g;
+                                const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
+                                *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
+                                    make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                                if (c4 == 0 && p.lse_out)
+                                    p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
+                            }
                         }
                         if (et == 0) p.counters[it.part_first] = 0;  // ready for the next launch
                     }

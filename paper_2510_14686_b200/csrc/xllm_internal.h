@@ -15,7 +15,7 @@ struct PlanTuning {
     int32_t tile_cost = 8;        // cost of one full KV tile block on the partition axis
     int32_t unit_overhead = 6;    // fixed cost of starting a unit (Q load, hand-off, output), same scale ...
     int32_t row_overhead = 8;     // ... plus this much for a full 16-row unit, in proportion to its rows
-    int32_t pieces_first = 0;     // 1: inside a CTA the pieces of split units run before the whole units (measured slower on B200)
+    int32_t pieces_first = 1;     // 1: inside a CTA the pieces of split units run before the whole units
     int32_t min_piece_tiles = 6;  // pieces of a split unit are at least this many tiles (swept on B200: 4..8 are within noise)
 };
 
@@ -59,7 +59,7 @@ inline int64_t tile_block_bytes(int32_t n_kv_heads, int32_t head_dim) { return n
 // ---- device-side records ------------------------------------------------------------------------------
 constexpr int32_t kMaxCtas = 160;  // upper bound on the persistent grid (B200: 148 SMs)
 
-constexpr int32_t kFuseMaxParts = 8;  // units split into at most this many pieces are merged inside the attention kernel
+constexpr int32_t kFuseMaxParts = 4;  // units split into at most this many pieces are merged inside the attention kernel
 
 struct DevItem {            // one work item, resolved on the host against the slot table (48 bytes)
     uint64_t kv;            // address of the item's KV head inside tile block 0 of the slot's range

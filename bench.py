@@ -5,8 +5,9 @@
     python bench.py --impl reference ...      # the fp64 CPU oracle on a bounded sample (reported baseline)
 
 One step = one pass of the whole hot path over one batch: map pages for the tokens about to be written,
-append the new K/V rows, partition the work, split-KV attention, LSE combine, then roll the sequence
-length back so that every step sees the named context lengths.  Prints ONE JSON line (rank 0).
+then one library call that appends the new K/V rows, partitions the work, runs the split-KV attention and the
+LSE merge (the append rides along in the attention launch), then roll the sequence length back so that every
+step sees the named context lengths.  Prints ONE JSON line (rank 0).
 
 Metric: KV tokens/s = sum of context lengths attended per step / step time; `value` is timed with CUDA
 events with all inputs resident in HBM, `e2e` through the same C-ABI calls with pinned HOST buffers for
@@ -233,12 +234,12 @@ class Replica:
         ctx, slots = self.ctx, self.slots[i % self.copies]
         q = self.q if q is None else q
         ctx.kv_map_pages_many(slots, self.kv)                              # a1: pages for the tokens about to be written
-        ctx.kv_append(slots, self.ql, self.k_new if k_new is None else k_new, self.v_new if v_new is None else v_new,
-                      self.stream)                                         # a2
-        if self.decode_only:                                               # a3 + a4 + a5
-            ctx.decode_attention(slots, q, self.out, None, self.s.scale, self.stream)
+        k_new = self.k_new if k_new is None else k_new
+        v_new = self.v_new if v_new is None else v_new
+        if self.decode_only:                                               # a2 + a3 + a4 + a5 in one call
+            ctx.append_decode_attention(slots, k_new, v_new, q, self.out, None, self.s.scale, self.stream)
         else:
-            ctx.verify_attention(slots, self.ql, q, self.out, None, self.s.scale, self.stream)
+            ctx.append_verify_attention(slots, self.ql, k_new, v_new, q, self.out, None, self.s.scale, self.stream)
         ctx.kv_set_len_many(slots, self.pre)                               # back to the named context lengths
 
     def step_e2e(self, i: int):

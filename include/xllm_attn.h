@@ -206,6 +206,20 @@ xllm_status xllm_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *s
 xllm_status xllm_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
                                   const void *q, void *out, float *lse_out, float scale, void *cuda_stream);
 
+/* Append and attend in one call: exactly xllm_kv_append(n_new = 1 per request, resp. n_new = q_lens) followed by
+ * xllm_decode_attention / xllm_verify_attention, but the new rows are written by the attention launch itself (the CTA
+ * that owns the last tiles of a (request, KV head) writes them before it fetches those tiles), which saves a launch
+ * and a dependent-kernel boundary per step ("write_kvcache" and attention of one decode step).  k_new, v_new: device
+ * bf16 [n_req, H_kv, D] resp. [sum q_lens, H_kv, D], request-major like q.  The target tokens must already be mapped
+ * (else NOT_MAPPED, nothing written).  When some request's rows do not fit one row group (H_q / H_kv * q_len > 16) the
+ * call falls back to two launches; the result is the same. */
+xllm_status xllm_append_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const void *k_new,
+                                         const void *v_new, const void *q, void *out, float *lse_out, float scale,
+                                         void *cuda_stream);
+xllm_status xllm_append_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
+                                         const void *k_new, const void *v_new, const void *q, void *out, float *lse_out,
+                                         float scale, void *cuda_stream);
+
 /* ---- decode attention without a context and without any allocation ------------------------------------------- */
 
 #define XLLM_STATIC_MAX_REQUESTS 64 /* requests per call of xllm_decode_attention_static */

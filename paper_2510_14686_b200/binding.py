@@ -94,6 +94,8 @@ EXPORTS = {
     "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
     "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_append_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_append_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_decode_attention_static": (ctypes.c_int32, [ctypes.c_int32, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                        _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
@@ -279,6 +281,16 @@ class Context:
         s, ql = _i32(slots), _i32(q_lens)
         self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(q), _ptr(out),
                                                _ptr(lse_out), scale, _stream(stream)))
+
+    def append_decode_attention(self, slots, k_new, v_new, q, out, lse_out=None, scale: float = 1.0, stream=None):
+        s = _i32(slots)
+        self._check(_lib.xllm_append_decode_attention(self._ctx, len(s), s.ctypes.data, _ptr(k_new), _ptr(v_new), _ptr(q),
+                                                      _ptr(out), _ptr(lse_out), scale, _stream(stream)))
+
+    def append_verify_attention(self, slots, q_lens, k_new, v_new, q, out, lse_out=None, scale: float = 1.0, stream=None):
+        s, ql = _i32(slots), _i32(q_lens)
+        self._check(_lib.xllm_append_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(k_new), _ptr(v_new),
+                                                      _ptr(q), _ptr(out), _ptr(lse_out), scale, _stream(stream)))
 
     def sync_check(self, stream=None):
         self._check(_lib.xllm_sync_check(self._ctx, _stream(stream)))

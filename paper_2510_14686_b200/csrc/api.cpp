@@ -73,6 +73,11 @@ struct xllm_ctx {
     std::vector<CombineDesc> combine;
     std::vector<int64_t> kv_lens;
     std::vector<uint8_t> seen;
+    std::vector<int32_t> ones_;
+    const int32_t *ones(int32_t n) {
+        if ((int32_t)ones_.size() < n) ones_.assign((size_t)n, 1);
+        return ones_.data();
+    }
 };
 
 namespace {
@@ -182,9 +187,13 @@ xllm_status check_slot_list(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, 
     return XLLM_OK;
 }
 
+// k_new / v_new non-null: the call first appends q_len new rows per request (fused into the attention launch when every
+// request's rows fit one row group, else by a separate append launch) and then attends over the grown ranges.
 xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
-                           void *out, float *lse_out, float scale, void *cuda_stream, const char *who) {
+                           void *out, float *lse_out, float scale, void *cuda_stream, const char *who,
+                           const void *k_new = nullptr, const void *v_new = nullptr) {
     if (!ctx) return XLLM_ERR_INVALID;
+    const bool with_append = k_new != nullptr || v_new != nullptr;
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context is host-only, no GPU work possible");
     xllm_status st = check_device_flag(ctx);
     if (st != XLLM_OK) return st;
@@ -195,13 +204,28 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q and out must be 16-byte aligned");
     if (!(scale > 0.f) || !std::isfinite(scale)) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": scale must be finite and > 0");
 
+    if (with_append && (!k_new || !v_new || (reinterpret_cast<uintptr_t>(k_new) & 15) || (reinterpret_cast<uintptr_t>(v_new) & 15)))
+        return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": k_new and v_new must be non-null and 16-byte aligned");
     ctx->kv_lens.resize((size_t)n_req);
     int64_t q_rows = 0;
+    bool one_group = ctx->tune.min_piece_tiles >= 2;  // fused append needs the last two tiles of a unit in one piece
     for (int32_t i = 0; i < n_req; ++i) {
         const int32_t ql = q_lens ? q_lens[i] : 1;
         const SlotRecord &s = ctx->xt->slot(slots[i]);
         if (ql < 1 || ql > ctx->cfg.max_q_len)
             return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q_len of request " + std::to_string(i) + " outside [1, max_q_len]");
+        if (with_append) {
+            if (s.kv_len + ql > ctx->cfg.max_seq_len)
+                return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(slots[i]) + " would exceed max_seq_len");
+            if (s.kv_len + ql > ctx->xt->mapped_tokens(slots[i]))
+                return fail(ctx, XLLM_ERR_NOT_MAPPED, std::string(who) + ": slot " + std::to_string(slots[i]) + " has pages for " +
+                                                          std::to_string(ctx->xt->mapped_tokens(slots[i])) + " tokens, needs " +
+                                                          std::to_string(s.kv_len + ql) + "; call xllm_kv_map_pages first");
+            if (ql * (ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads) > kMaxRows) one_group = false;
+            ctx->kv_lens[(size_t)i] = s.kv_len + ql;
+            q_rows += ql;
+            continue;
+        }
         if (s.kv_len < ql)
             return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(slots[i]) + " holds " +
                                                    std::to_string(s.kv_len) + " tokens, fewer than q_len " + std::to_string(ql));
@@ -235,6 +259,22 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
             combine.push_back({it.part_first, it.n_parts, q_row0[(size_t)it.req] + it.q_tok0, it.kv_head * G + it.g0, it.n_q_tok,
                                it.n_g});
 
+    // Fused append: the piece that holds a unit's last tile must also hold the tile of the request's first new token.
+    // It pays when a CTA has few work items (the copy runs at the start of the kernel on the warps that later finish
+    // items); with many short items per CTA a separate append launch is faster (measured on B200: break-even ~8-10).
+    bool fuse = with_append && one_group && n_items <= ctx->tune.fuse_max_items_per_cta * ctx->sm_count;
+    if (fuse) {
+        for (const xllm_work_item &w : ctx->items) {
+            const int32_t ql = q_lens ? q_lens[w.req] : 1;
+            const int64_t kv = ctx->kv_lens[(size_t)w.req];
+            if (w.tile_end == (kv + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS && (int64_t)w.tile_begin * XLLM_TILE_TOKENS > kv - ql) fuse = false;
+        }
+    }
+    if (with_append && !fuse) {  // two launches: the plan above already counts the new tokens
+        const xllm_status as = xllm_kv_append(ctx, n_req, slots, q_lens ? q_lens : ctx->ones(n_req), k_new, v_new, cuda_stream);
+        if (as != XLLM_OK) return as;
+    }
+
     int idx;
     int e = acquire_stage(ctx, &idx);
     if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
@@ -255,13 +295,15 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         di[i].partial_idx = w.partial_idx;
         di[i].tile_begin = w.tile_begin;
         di[i].tile_end = w.tile_end;
-        di[i].kv_end = (int32_t)s.kv_len - ql + w.q_tok0 + w.n_q_tok;
+        const int64_t kv_now = ctx->kv_lens[(size_t)w.req];  // tokens in the range when the kernel reads it
+        di[i].kv_end = (int32_t)kv_now - ql + w.q_tok0 + w.n_q_tok;
         di[i].head0 = (int16_t)(w.kv_head * G + w.g0);
         di[i].n_q_tok = (uint8_t)w.n_q_tok;
         di[i].n_g = (uint8_t)w.n_g;
         di[i].part_first = w.part_first;
         di[i].n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
-        di[i].pad[0] = di[i].pad[1] = 0;
+        di[i].new_row = q_row0[(size_t)w.req];
+        di[i].n_new = (fuse && w.tile_end == (kv_now + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS) ? ql : 0;
     }
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
 
@@ -271,6 +313,8 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     AttnLaunch al{};
     al.items = reinterpret_cast<const DevItem *>(d + off_items);
     al.q = q;
+    al.k_new = fuse ? k_new : nullptr;
+    al.v_new = fuse ? v_new : nullptr;
     al.out = out;
     al.lse_out = lse_out;
     al.part_o = ctx->d_part_o;
@@ -308,7 +352,12 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         ++ctx->st.kernel_launches;
     }
     finish_launch(ctx, idx, stream);
-    for (int32_t i = 0; i < n_req; ++i) ctx->xt->slot(slots[i]).last_use = ctx->seq;
+    for (int32_t i = 0; i < n_req; ++i) {
+        SlotRecord &s = ctx->xt->slot(slots[i]);
+        s.last_use = ctx->seq;
+        if (fuse) s.kv_len = ctx->kv_lens[(size_t)i];  // the attention launch wrote the new rows
+    }
+    if (fuse) ctx->st.tokens_appended += q_rows;
     ++ctx->st.attention_calls;
     ctx->st.work_items += n_items;
     ctx->st.partial_items += n_partials;
@@ -669,6 +718,20 @@ xllm_status xllm_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *s
                                   void *out, float *lse_out, float scale, void *cuda_stream) {
     if (ctx && !q_lens) return fail(ctx, XLLM_ERR_INVALID, "verify_attention: q_lens must be non-null");
     return attention_impl(ctx, n_req, slots, q_lens, q, out, lse_out, scale, cuda_stream, "verify_attention");
+}
+
+xllm_status xllm_append_decode_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const void *k_new, const void *v_new,
+                                         const void *q, void *out, float *lse_out, float scale, void *cuda_stream) {
+    if (ctx && (!k_new || !v_new)) return fail(ctx, XLLM_ERR_INVALID, "append_decode_attention: k_new and v_new must be non-null");
+    return attention_impl(ctx, n_req, slots, nullptr, q, out, lse_out, scale, cuda_stream, "append_decode_attention", k_new, v_new);
+}
+
+xllm_status xllm_append_verify_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
+                                         const void *k_new, const void *v_new, const void *q, void *out, float *lse_out,
+                                         float scale, void *cuda_stream) {
+    if (ctx && (!q_lens || !k_new || !v_new))
+        return fail(ctx, XLLM_ERR_INVALID, "append_verify_attention: q_lens, k_new and v_new must be non-null");
+    return attention_impl(ctx, n_req, slots, q_lens, q, out, lse_out, scale, cuda_stream, "append_verify_attention", k_new, v_new);
 }
 
 xllm_status xllm_plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,

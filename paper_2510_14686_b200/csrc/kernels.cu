@@ -66,7 +66,7 @@ struct Cfg {
     static constexpr int kOffQ = kOffP + 2 * 2 * kMaxRows * kPPitch;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
     static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(DevItem);
-    static constexpr int kNumBars = 2 * kHalfStages + 7;
+    static constexpr int kNumBars = 2 * kHalfStages + 8;
     static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast
     static constexpr int kSmemBytes = kOffFlags + 16;
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
@@ -311,6 +311,47 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
     if (lane == 0) mbar_arrive(bar_v_empty);  // this warp is done with the V half
 }
 
+// Fused append ("write_kvcache" inside the attention launch): an item with n_new > 0 owns the last tiles of its
+// (request, KV head) and nobody else reads them, so this CTA writes the step's new K/V rows into the range itself.
+// All items of a batch are handled in one flat loop (item, 16-byte chunk) whose loads are issued four at a time before
+// their stores: the copy is a chain of HBM round trips otherwise.  `tid`/`nthreads`: the threads sharing the copy.
+// The caller fences (generic -> async proxy) and synchronises before the tiles are fetched.
+template <int D>
+__device__ __forceinline__ void append_new_rows(const DevItem *sitems, const DevItem &first, bool use_first, int nb,
+                                                const AttnLaunch &p, int64_t tile_block, int tid, int nthreads) {
+    constexpr int cpr = D / 8;  // 16-byte chunks per head row
+    int max_new = 0;
+    for (int i = 0; i < nb; ++i) max_new = max(max_new, (use_first && i == 0) ? first.n_new : sitems[i].n_new);
+    if (max_new == 0) return;
+    const int stride = 2 * max_new * cpr;  // flat index space per item
+    const int total = nb * stride;
+    constexpr int kU = 4;
+    for (int f0 = tid; f0 < total; f0 += kU * nthreads) {
+        uint4 val[kU];
+        char *dst[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int f = f0 + u * nthreads;
+            dst[u] = nullptr;
+            if (f >= total) continue;
+            const int i = f / stride, c = f - i * stride;
+            const DevItem &it = (use_first && i == 0) ? first : sitems[i];
+            if (c >= 2 * it.n_new * cpr) continue;
+            const int which = c / (it.n_new * cpr), r = (c / cpr) % it.n_new, ch = c % cpr;
+            const int h = it.head0 / (p.n_q_heads / p.n_kv_heads);
+            val[u] = static_cast<const uint4 *>(which ? p.v_new : p.k_new)[((int64_t)(it.new_row + r) * p.n_kv_heads + h) * cpr + ch];
+            const int64_t pos = (int64_t)it.kv_end - it.n_new + r;  // the item's row group covers all query tokens: kv_end = kv_len
+            const int64_t blk = pos / T;
+            const int tr = (int)(pos % T);
+            dst[u] = const_cast<char *>(reinterpret_cast<const char *>(it.kv)) + blk * tile_block + (int64_t)which * Cfg<D>::kHalfTile +
+                     (ch >> 3) * kPanelBytes + tr * 128 + (((ch & 7) ^ (tr & 7)) << 4);
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+            if (dst[u]) *reinterpret_cast<uint4 *>(dst[u]) = val[u];
+    }
+}
+
 template <int D, bool TRACE>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnLaunch p) {
     using C = Cfg<D>;
@@ -326,6 +367,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const uint32_t bar_mfull = bar_qempty + 16;                       // group states of an item written (8 warps)
     const uint32_t bar_mempty = bar_mfull + 8;                        // ... and read by the epilogue (3 warps)
     const uint32_t bar_items = bar_mempty + 8;                        // first batch of item records is in shared memory
+    const uint32_t bar_append = bar_items + 8;                        // first batch's new K/V rows are in their ranges
     const unsigned long long t_start = TRACE ? clock64() : 0ull;
     const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
 
@@ -342,6 +384,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         mbar_init(bar_mfull, kConsumerWarps);
         mbar_init(bar_mempty, kEpilogueWarps);
         mbar_init(bar_items, kEpilogueWarps);
+        mbar_init(bar_append, kEpilogueWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -370,13 +413,29 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_items);
+                if (p.k_new) {  // fused append: these warps are idle until the first item finishes
+                    mbar_wait(bar_items, 0, abort_flag, p.error_flag, 8);
+                    append_new_rows<D>(sitems, p.first_item[blockIdx.x], true, nb, p, (int64_t)p.n_kv_heads * 2 * C::kHalfTile,
+                                       tid - kEpilogueWarp0 * 32, kEpilogueThreads);
+                    __threadfence();
+                    asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores before the bulk copies that read them
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_append);
+                }
             }
         } else {
             __syncthreads();  // everyone is done with the previous batch's records
             for (int i = tid; i < nb * 3; i += kThreads)
                 reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
             __syncthreads();
+            if (p.k_new) {
+                append_new_rows<D>(sitems, sitems[0], false, nb, p, (int64_t)p.n_kv_heads * 2 * C::kHalfTile, tid, kThreads);
+                __threadfence();
+                asm volatile("fence.proxy.async;" ::: "memory");
+                __syncthreads();
+            }
         }
+        bool append_done = !first_batch || !p.k_new;  // producer: already waited for the appended rows of this batch
         // record of item i of this batch; waits (once) for the fetch above before the first use of shared memory
         bool items_ready = !first_batch;
         auto item_at = [&](int i) -> DevItem {
@@ -390,9 +449,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 
         if (warp == kProducerWarp) {
             // ================= producer =================
-            if (lane == 0) {
-                for (int i = 0; i < nb; ++i) {
-                    const DevItem it = item_at(i);
+            for (int i = 0; i < nb; ++i) {
+                const DevItem it = item_at(i);
+                if (lane == 0) {
                     const int n_rows = it.n_q_tok * it.n_g;
                     const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
                     if (mbar_wait(bar_qempty + qb * 8, qph ^ 1, abort_flag, p.error_flag, 1)) {
@@ -409,6 +468,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                         const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);
                         const uint32_t bytes = rows * 128;
                         const char *src = kv + (int64_t)tile * tile_block;
+                        if (it.n_new > 0 && !append_done && tile * T + T > it.kv_end - it.n_new) {
+                            // this tile holds rows the launch itself appends: wait until they are in the range
+                            mbar_wait(bar_append, 0, abort_flag, p.error_flag, 9);
+                            append_done = true;
+                        }
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {  // K half, then V half
                             uint32_t hs, ph;

@@ -162,7 +162,7 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
         d.n_g = (uint8_t)w.n_g;
         d.part_first = w.part_first;
         d.n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
-        d.pad[0] = d.pad[1] = 0;
+        d.new_row = d.n_new = 0;
     }
 
     // ---- stage the lists in the scratch array (copies from pageable memory are staged by the driver before the

@@ -16,7 +16,8 @@ struct PlanTuning {
     int32_t unit_overhead = 6;    // fixed cost of starting a unit (Q load, hand-off, output), same scale ...
     int32_t row_overhead = 8;     // ... plus this much for a full 16-row unit, in proportion to its rows
     int32_t pieces_first = 1;     // 1: inside a CTA the pieces of split units run before the whole units
-    int32_t min_piece_tiles = 6;  // pieces of a split unit are at least this many tiles (swept on B200: 4..8 are within noise)
+    int32_t fuse_max_items_per_cta = 8;  // append rides along in the attention launch up to this many work items per CTA
+    int32_t min_piece_tiles = 4;  // pieces of a split unit are at least this many tiles (swept on B200: 2..8 are within noise; >= 2 required)
 };
 
 struct PlanUnit {  // one (request, KV head, row group) on the planner's cost axis
@@ -71,7 +72,8 @@ struct DevItem {            // one work item, resolved on the host against the s
     uint8_t n_q_tok, n_g;   // rows = n_q_tok * n_g <= kMaxRows
     int32_t part_first;     // partial slot of the unit's first piece (also the index of the unit's arrival counter)
     int32_t n_parts;        // pieces of the unit if the last piece to finish merges them in-kernel; 0 = combine kernel
-    int32_t pad[2];
+    int32_t new_row;        // fused append: first row of the request's new tokens in k_new / v_new ...
+    int32_t n_new;          // ... and how many this item must write into the range before reading its last tiles (else 0)
 };
 static_assert(sizeof(DevItem) == 48, "DevItem layout");
 
@@ -98,6 +100,7 @@ struct AppendLaunch {
 struct AttnLaunch {
     const DevItem *items;         // device, grouped by CTA
     const void *q;
+    const void *k_new, *v_new;    // fused append: rows [sum n_new, H_kv, D] of the step's new tokens, else null
     void *out;
     float *lse_out;               // may be null
     float *part_o;                // [n_partials][kMaxRows][D] fp32

@@ -449,9 +449,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 
         if (warp == kProducerWarp) {
             // ================= producer =================
-            for (int i = 0; i < nb; ++i) {
+            for (int i = 0; i < nb && lane == 0; ++i) {  // one elected lane issues every copy; the others wait below
                 const DevItem it = item_at(i);
-                if (lane == 0) {
+                {
                     const int n_rows = it.n_q_tok * it.n_g;
                     const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
                     if (mbar_wait(bar_qempty + qb * 8, qph ^ 1, abort_flag, p.error_flag, 1)) {

@@ -754,22 +754,39 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 template <int D>
 __global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
     grid_launch_dependents();
-    grid_dependency_wait();  // the partial results come from the attention kernel launched just before
-    const CombineDesc d = p.descs[blockIdx.x];
+    const CombineDesc d = p.descs[blockIdx.x];  // written by the host before the launch: fetched while the attention kernel drains
+    grid_dependency_wait();                     // the partial results come from the attention kernel launched just before
     const int row = blockIdx.y;
     if (row >= d.n_q_tok * d.n_g) return;
     const int col = threadIdx.x;
+    // Two passes over the pieces, eight at a time with all loads of a batch issued before any is used (a piece sits
+    // in L2; serial round trips would dominate this tiny kernel).  Pass 1: the row's maximum; pass 2: weighted sum.
+    constexpr int kB = 8;
     float M = -INFINITY;
-    for (int s = 0; s < d.n_parts; ++s) M = fmaxf(M, p.part_lse[(int64_t)(d.partial_begin + s) * kMaxRows + row]);
+    for (int s0 = 0; s0 < d.n_parts; s0 += kB) {
+        float ls[kB];
+#pragma unroll
+        for (int j = 0; j < kB; ++j)
+            ls[j] = (s0 + j < d.n_parts) ? p.part_lse[(int64_t)(d.partial_begin + s0 + j) * kMaxRows + row] : -INFINITY;
+#pragma unroll
+        for (int j = 0; j < kB; ++j) M = fmaxf(M, ls[j]);
+    }
+    const float Ms = (M == -INFINITY) ? 0.f : M;
     float acc = 0.f, W = 0.f;
-    if (M != -INFINITY) {
-        for (int s = 0; s < d.n_parts; ++s) {
-            const int64_t pi = d.partial_begin + s;
-            const float ls = p.part_lse[pi * kMaxRows + row];
-            if (ls == -INFINITY) continue;  // a piece in which this row saw no key
-            const float w = exp2f(ls - M);
+    for (int s0 = 0; s0 < d.n_parts; s0 += kB) {
+        float ls[kB], v[kB];
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {
+            const int64_t pi = d.partial_begin + s0 + j;
+            const bool ok = s0 + j < d.n_parts;
+            ls[j] = ok ? p.part_lse[pi * kMaxRows + row] : -INFINITY;
+            v[j] = ok ? p.part_o[(pi * kMaxRows + row) * D + col] : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < kB; ++j) {  // piece order: repeatable bit for bit
+            const float w = exp2f(ls[j] - Ms);  // 0 for a piece in which this row saw no key, and for padding
             W += w;
-            acc += w * p.part_o[(pi * kMaxRows + row) * D + col];
+            acc += w * v[j];
         }
     }
     const int ti = row / d.n_g, gi = row - ti * d.n_g;

@@ -80,6 +80,8 @@ typedef struct {
     double append_kernel_ms;      /* same for the append kernel */
     int64_t combine_launches, append_launches;
     int64_t kernel_launches;      /* kernels of this library launched so far (append, gather, attention, combine) */
+    int64_t pages_premapped_total; /* of pages_mapped_total, pages mapped by the pre-mapping worker thread */
+    double premap_host_us;        /* of map_host_us, time spent in the worker thread (hidden from the caller) */
     int32_t sm_count;             /* CTAs of the persistent attention grid */
     int32_t reserved;
 } xllm_stats;
@@ -145,6 +147,18 @@ xllm_status xllm_kv_map_pages(xllm_ctx *ctx, int32_t slot, int64_t min_tokens);
 /* The same for n_req slots in one call (one scheduler step): slot slots[i] is grown to min_tokens[i].  Stops at
  * the first failure; slots before it keep their new pages. */
 xllm_status xllm_kv_map_pages_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens);
+
+/* Asynchronous pre-mapping ("Low Overhead Allocation": while the current token is decoded, the pages the next
+ * token needs are mapped in the background).  Queues the growth of slots[i] to min_tokens[i] and returns at once; a
+ * worker thread of the context (started on first use) does what xllm_kv_map_pages would do, while the caller goes
+ * on -- typically right after the step's kernels were launched, so that the driver's map latency overlaps the GPU
+ * work.  A later xllm_kv_map_pages on the slot finds the pages there (or maps what is still missing).  Jobs for
+ * slots released in the meantime are dropped.  Every entry point of a context is serialised against the worker by
+ * one lock, so any call may be made while jobs are pending. */
+xllm_status xllm_kv_premap_async(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens);
+/* Block until every queued job has run; returns (and clears) the first failure of the background mapping, with its
+ * message in xllm_last_error (e.g. XLLM_ERR_OOM_PHYS). */
+xllm_status xllm_kv_premap_wait(xllm_ctx *ctx);
 
 /* End a request.  mode 0: keep the pages mapped in the range, Status = Reusable, for the next request
  * that takes the slot over; mode 1: unmap them back to the Free stack (waits for work in flight on the

@@ -51,7 +51,7 @@ class Stats(ctypes.Structure):
                 ("partial_items", ctypes.c_int64), ("attn_launches", ctypes.c_int64), ("attn_kernel_ms", ctypes.c_double),
                 ("combine_kernel_ms", ctypes.c_double), ("append_kernel_ms", ctypes.c_double),
                 ("combine_launches", ctypes.c_int64), ("append_launches", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
-                ("sm_count", ctypes.c_int32),
+                ("pages_premapped_total", ctypes.c_int64), ("premap_host_us", ctypes.c_double), ("sm_count", ctypes.c_int32),
                 ("reserved", ctypes.c_int32)]
 
     def as_dict(self):
@@ -83,6 +83,8 @@ EXPORTS = {
     "xllm_kv_map_pages": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
     "xllm_kv_map_pages_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp]),
     "xllm_kv_set_len_many": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp]),
+    "xllm_kv_premap_async": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp]),
+    "xllm_kv_premap_wait": (ctypes.c_int32, [_ctxp]),
     "xllm_kv_release": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int32]),
     "xllm_kv_set_len": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64]),
     "xllm_kv_slot_info": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.POINTER(SlotInfo)]),
@@ -229,6 +231,13 @@ class Context:
     def kv_set_len_many(self, slots, kv_lens):
         s, t = _i32(slots), _i64(kv_lens)
         self._check(_lib.xllm_kv_set_len_many(self._ctx, len(s), s.ctypes.data, t.ctypes.data))
+
+    def kv_premap_async(self, slots, min_tokens):
+        s, t = _i32(slots), _i64(min_tokens)
+        self._check(_lib.xllm_kv_premap_async(self._ctx, len(s), s.ctypes.data, t.ctypes.data))
+
+    def kv_premap_wait(self):
+        self._check(_lib.xllm_kv_premap_wait(self._ctx))
 
     def kv_release(self, slot: int, mode: int = 0):
         self._check(_lib.xllm_kv_release(self._ctx, slot, mode))

@@ -6,7 +6,11 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <condition_variable>
+#include <deque>
 #include <memory>
+#include <mutex>
+#include <thread>
 #include <string>
 #include <vector>
 
@@ -36,7 +40,26 @@ namespace xllm {
 void set_init_error(const char *msg) { g_init_error = msg ? msg : ""; }
 }  // namespace xllm
 
+struct PremapJob {
+    int32_t slot;
+    int64_t min_tokens;
+};
+
 struct xllm_ctx {
+    // One lock serialises every entry point and the pre-mapping worker (recursive: the fused append falls back to
+    // xllm_kv_append from inside an attention call).
+    std::recursive_mutex mu;
+    // asynchronous pre-mapping: jobs queued by xllm_kv_premap_async, executed by one worker thread
+    std::thread worker;
+    std::mutex qmu;
+    std::condition_variable qcv, qidle;
+    std::deque<PremapJob> queue;
+    bool worker_busy = false, worker_stop = false;
+    xllm_status premap_status = XLLM_OK;
+    std::string premap_err;
+    int64_t pages_premapped = 0;
+    double premap_us = 0.0;
+
     xllm_config cfg{};
     std::unique_ptr<XTensor> xt;
     bool host_only = false;
@@ -79,6 +102,8 @@ struct xllm_ctx {
         return ones_.data();
     }
 };
+
+#define XLLM_LOCK(ctx) std::lock_guard<std::recursive_mutex> xllm_lock_((ctx)->mu)
 
 namespace {
 
@@ -187,12 +212,59 @@ xllm_status check_slot_list(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, 
     return XLLM_OK;
 }
 
+// Pre-mapping worker: maps pages for queued (slot, min_tokens) jobs while the caller's thread goes on -- typically while
+// the current step's kernels run ("Asynchronous Pre-mapping": the pages the next token needs are mapped during the
+// current decode, so the map latency is hidden).
+void premap_worker(xllm_ctx *ctx) {
+    if (!ctx->host_only) cudaSetDevice(ctx->cfg.device);  // driver calls need the device's primary context current
+    for (;;) {
+        PremapJob job;
+        {
+            std::unique_lock<std::mutex> lk(ctx->qmu);
+            ctx->worker_busy = false;
+            if (ctx->queue.empty()) ctx->qidle.notify_all();
+            ctx->qcv.wait(lk, [ctx] { return ctx->worker_stop || !ctx->queue.empty(); });
+            if (ctx->worker_stop) return;
+            job = ctx->queue.front();
+            ctx->queue.pop_front();
+            ctx->worker_busy = true;
+        }
+        std::lock_guard<std::recursive_mutex> lk(ctx->mu);
+        if (!ctx->xt->valid_slot(job.slot) || !ctx->xt->slot(job.slot).live) continue;  // finished meanwhile: nothing to do
+        xllm_stats before{}, after{};
+        ctx->xt->fill_stats(&before);
+        std::string err;
+        const xllm_status st = ctx->xt->map_pages(job.slot, job.min_tokens, &err);
+        ctx->xt->fill_stats(&after);
+        ctx->pages_premapped += after.pages_mapped_total - before.pages_mapped_total;
+        ctx->premap_us += after.map_host_us - before.map_host_us;
+        if (st != XLLM_OK) {
+            std::lock_guard<std::mutex> ql(ctx->qmu);
+            if (ctx->premap_status == XLLM_OK) {
+                ctx->premap_status = st;
+                ctx->premap_err = "pre-mapping slot " + std::to_string(job.slot) + ": " + err;
+            }
+        }
+    }
+}
+
+void stop_worker(xllm_ctx *ctx) {
+    if (!ctx->worker.joinable()) return;
+    {
+        std::lock_guard<std::mutex> lk(ctx->qmu);
+        ctx->worker_stop = true;
+    }
+    ctx->qcv.notify_all();
+    ctx->worker.join();
+}
+
 // k_new / v_new non-null: the call first appends q_len new rows per request (fused into the attention launch when every
 // request's rows fit one row group, else by a separate append launch) and then attends over the grown ranges.
 xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
                            void *out, float *lse_out, float scale, void *cuda_stream, const char *who,
                            const void *k_new = nullptr, const void *v_new = nullptr) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     const bool with_append = k_new != nullptr || v_new != nullptr;
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context is host-only, no GPU work possible");
     xllm_status st = check_device_flag(ctx);
@@ -475,6 +547,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
 
 xllm_status xllm_shutdown(xllm_ctx *ctx) {
     if (!ctx) return XLLM_ERR_INVALID;
+    stop_worker(ctx);
     if (!ctx->host_only) {
         cudaSetDevice(ctx->cfg.device);
         cudaDeviceSynchronize();
@@ -505,6 +578,7 @@ const char *xllm_last_error(const xllm_ctx *ctx) { return ctx ? ctx->err.c_str()
 
 xllm_status xllm_sync_check(xllm_ctx *ctx, void *cuda_stream) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (ctx->host_only) return XLLM_OK;
     const cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return cuda_fail(ctx, "cudaStreamSynchronize", (int)e);
@@ -513,16 +587,19 @@ xllm_status xllm_sync_check(xllm_ctx *ctx, void *cuda_stream) {
 
 xllm_status xllm_kv_reserve(xllm_ctx *ctx, int64_t max_seq_len, int64_t expected_tokens, int32_t *slot_out) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     return ctx->xt->reserve(max_seq_len, expected_tokens, slot_out, &ctx->err);
 }
 
 xllm_status xllm_kv_map_pages(xllm_ctx *ctx, int32_t slot, int64_t min_tokens) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     return ctx->xt->map_pages(slot, min_tokens, &ctx->err);
 }
 
 xllm_status xllm_kv_map_pages_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (n_req < 0 || !slots || !min_tokens) return fail(ctx, XLLM_ERR_INVALID, "map_pages_many: null argument");
     for (int32_t i = 0; i < n_req; ++i) {
         const xllm_status st = ctx->xt->map_pages(slots[i], min_tokens[i], &ctx->err);
@@ -531,13 +608,49 @@ xllm_status xllm_kv_map_pages_many(xllm_ctx *ctx, int32_t n_req, const int32_t *
     return XLLM_OK;
 }
 
+xllm_status xllm_kv_premap_async(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *min_tokens) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    if (n_req < 0 || (n_req > 0 && (!slots || !min_tokens))) {
+        XLLM_LOCK(ctx);
+        return fail(ctx, XLLM_ERR_INVALID, "premap_async: null argument");
+    }
+    {
+        std::lock_guard<std::mutex> lk(ctx->qmu);
+        for (int32_t i = 0; i < n_req; ++i) ctx->queue.push_back({slots[i], min_tokens[i]});
+        if (!ctx->worker.joinable()) ctx->worker = std::thread(premap_worker, ctx);  // started on first use
+    }
+    ctx->qcv.notify_one();
+    return XLLM_OK;
+}
+
+xllm_status xllm_kv_premap_wait(xllm_ctx *ctx) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    xllm_status st;
+    std::string err;
+    {
+        std::unique_lock<std::mutex> lk(ctx->qmu);
+        ctx->qidle.wait(lk, [ctx] { return ctx->queue.empty() && !ctx->worker_busy; });
+        st = ctx->premap_status;
+        err = ctx->premap_err;
+        ctx->premap_status = XLLM_OK;
+        ctx->premap_err.clear();
+    }
+    if (st != XLLM_OK) {
+        XLLM_LOCK(ctx);
+        return fail(ctx, st, err);
+    }
+    return XLLM_OK;
+}
+
 xllm_status xllm_kv_release(xllm_ctx *ctx, int32_t slot, int32_t mode) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     return ctx->xt->release(slot, mode, &ctx->err);
 }
 
 xllm_status xllm_kv_set_len(xllm_ctx *ctx, int32_t slot, int64_t kv_len) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "set_len: slot is not live");
     if (kv_len < 0 || kv_len > ctx->xt->mapped_tokens(slot) || kv_len > ctx->cfg.max_seq_len)
         return fail(ctx, XLLM_ERR_INVALID, "set_len: kv_len must lie in [0, mapped tokens]");
@@ -547,6 +660,7 @@ xllm_status xllm_kv_set_len(xllm_ctx *ctx, int32_t slot, int64_t kv_len) {
 
 xllm_status xllm_kv_set_len_many(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int64_t *kv_lens) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (n_req < 0 || !slots || !kv_lens) return fail(ctx, XLLM_ERR_INVALID, "set_len_many: null argument");
     for (int32_t i = 0; i < n_req; ++i) {
         if (!ctx->xt->valid_slot(slots[i]) || !ctx->xt->slot(slots[i]).live)
@@ -560,6 +674,7 @@ xllm_status xllm_kv_set_len_many(xllm_ctx *ctx, int32_t n_req, const int32_t *sl
 
 xllm_status xllm_kv_slot_info(const xllm_ctx *ctx, int32_t slot, xllm_slot_info *info) {
     if (!ctx || !info || !ctx->xt->valid_slot(slot)) return XLLM_ERR_INVALID;
+    XLLM_LOCK(const_cast<xllm_ctx *>(ctx));
     const SlotRecord &s = ctx->xt->slot(slot);
     info->base = s.base;
     info->va_bytes = ctx->xt->va_bytes();
@@ -575,6 +690,7 @@ xllm_status xllm_kv_slot_info(const xllm_ctx *ctx, int32_t slot, xllm_slot_info 
 xllm_status xllm_kv_page_of(const xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int32_t *page_pos, int32_t *page_id,
                             int64_t *in_page_offset) {
     if (!ctx || !ctx->xt->valid_slot(slot) || byte_offset < 0 || byte_offset >= ctx->xt->va_bytes()) return XLLM_ERR_INVALID;
+    XLLM_LOCK(const_cast<xllm_ctx *>(ctx));
     const SlotRecord &s = ctx->xt->slot(slot);
     const int64_t pos = byte_offset / ctx->xt->page_bytes();
     if (pos >= (int64_t)s.pages.size()) return XLLM_ERR_NOT_MAPPED;
@@ -586,6 +702,7 @@ xllm_status xllm_kv_page_of(const xllm_ctx *ctx, int32_t slot, int64_t byte_offs
 
 xllm_status xllm_debug_read_slot(xllm_ctx *ctx, int32_t slot, int64_t byte_offset, int64_t nbytes, void *host_dst) {
     if (!ctx || !host_dst) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_slot: host-only context");
     if (!ctx->xt->valid_slot(slot) || byte_offset < 0 || nbytes < 0) return fail(ctx, XLLM_ERR_INVALID, "debug_read_slot: bad arguments");
     const SlotRecord &s = ctx->xt->slot(slot);
@@ -598,6 +715,7 @@ xllm_status xllm_debug_read_slot(xllm_ctx *ctx, int32_t slot, int64_t byte_offse
 
 xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_offset, int64_t nbytes, void *host_dst) {
     if (!ctx || !host_dst) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_page: host-only context");
     const int64_t pb = ctx->xt->page_bytes();
     if (page_id < 0 || page_id >= (int32_t)ctx->xt->pages().size() || byte_offset < 0 || nbytes < 0 || byte_offset + nbytes > pb)
@@ -623,6 +741,7 @@ xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_of
 
 xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max_words, int32_t *n_words_out) {
     if (!ctx || !host_dst || !n_words_out) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (!ctx->d_trace) return fail(ctx, XLLM_ERR_UNSUPPORTED, "debug_read_trace: start the process with XLLM_TRACE=1 to collect a trace");
     const int32_t n = std::min(max_words, ctx->sm_count * kTraceWords);
     cudaError_t e = cudaDeviceSynchronize();
@@ -635,6 +754,7 @@ xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max
 xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new, const void *k_new,
                            const void *v_new, void *cuda_stream) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "append: context is host-only, no GPU work possible");
     xllm_status st = check_device_flag(ctx);
     if (st != XLLM_OK) return st;
@@ -689,6 +809,7 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
 xllm_status xllm_kv_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out,
                            void *cuda_stream) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "gather: context is host-only, no GPU work possible");
     if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "gather: slot is not live");
     if (!k_out || !v_out || (reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
@@ -753,14 +874,18 @@ xllm_status xllm_plan_partition(int32_t n_req, const int64_t *kv_lens, const int
 xllm_status xllm_get_stats(const xllm_ctx *ctx_c, xllm_stats *stats) {
     if (!ctx_c || !stats) return XLLM_ERR_INVALID;
     xllm_ctx *ctx = const_cast<xllm_ctx *>(ctx_c);
+    XLLM_LOCK(ctx);
     if (!ctx->host_only) resolve_timings(ctx);
     ctx->xt->fill_stats(&ctx->st);
+    ctx->st.pages_premapped_total = ctx->pages_premapped;
+    ctx->st.premap_host_us = ctx->premap_us;
     *stats = ctx->st;
     return XLLM_OK;
 }
 
 xllm_status xllm_set_profiling(xllm_ctx *ctx, int32_t on) {
     if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
     ctx->profiling = on != 0 && !ctx->host_only;
     return XLLM_OK;
 }

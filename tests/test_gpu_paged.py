@@ -87,3 +87,45 @@ def test_full_scenario_256_requests_ten_steps(binding):
     print(f"paged: worst max-abs {worst[0]:.2e} mean-abs {worst[1]:.2e}; mapped {st.pages_mapped_total} "
           f"unmapped {st.pages_unmapped_total} reused {st.pages_reused_total}; map {st.map_host_us:.0f} us unmap {st.unmap_host_us:.0f} us")
     assert st.pages_reused_total > 0 and st.pages_unmapped_total > 0
+
+
+def test_premap_async_hides_the_driver_map_latency(binding):
+    """The pages the next tokens need are mapped by the worker thread while the GPU runs the current step; the map call
+    on the critical path then finds them in place."""
+    import time
+
+    import gpu_harness as gh
+
+    batch = wl.custom_batch(515, 32, 8, 128, [500] * 64)             # 64 requests just below a page boundary (512 tokens)
+    s = batch.shape
+    with gh.make_ctx(binding, s, 64, 4096, [2048] * 64) as ctx:
+        slots = np.array(gh.load_requests(ctx, batch.requests), np.int32)
+        q = gh.dev_bits(np.concatenate([r.q for r in batch.requests]))
+        out = torch.zeros_like(q)
+        grow1, grow2 = np.full(64, 1024, np.int64), np.full(64, 1536, np.int64)
+        # (a) synchronous: 64 pages mapped on the critical path
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ctx.kv_map_pages_many(slots, grow1)
+        t_sync = (time.perf_counter() - t0) * 1e6
+        # (b) pre-mapped while a decode step runs on the GPU
+        ctx.decode_attention(slots, q, out, None, s.scale)
+        ctx.kv_premap_async(slots, grow2)
+        ctx.sync_check()                                            # the step's result is awaited anyway
+        ctx.kv_premap_wait()
+        t0 = time.perf_counter()
+        ctx.kv_map_pages_many(slots, grow2)                           # nothing left to do
+        t_fore = (time.perf_counter() - t0) * 1e6
+        st = ctx.get_stats()
+        assert st.pages_premapped_total == 64 and st.pages_mapped_total == 64 * 3
+        assert all(ctx.kv_slot_info(int(sl)).mapped_tokens >= 1536 for sl in slots)
+        print(f"map 64 pages on the critical path: {t_sync:.0f} us; after pre-mapping: {t_fore:.1f} us "
+              f"(worker spent {st.premap_host_us:.0f} us in the driver)")
+        assert t_fore < 0.2 * t_sync
+        # the pre-mapped pages are usable: append into them and attend
+        extra = wl.custom_batch(516, 32, 8, 128, [600] * 64)
+        k = gh.dev_bits(np.concatenate([r.k for r in extra.requests]))
+        ctx.kv_append(slots, np.full(64, 600, np.int32), k, k)
+        ctx.decode_attention(slots, q, out, None, s.scale)
+        ctx.sync_check()
+        assert ctx.kv_slot_info(int(slots[0])).kv_len == 1100

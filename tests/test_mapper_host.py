@@ -136,3 +136,54 @@ def test_eager_pool_creation_failure_is_reported(binding):
     with pytest.raises(binding.XllmError) as e:
         make(binding, fault_inject=5)
     assert e.value.status == binding.ERR_OOM_PHYS
+
+
+# ---- asynchronous pre-mapping (worker thread), host-only context -------------------------------------------
+def test_premap_async_maps_in_the_background(binding):
+    ctx, model = make(binding, n_pages=32, slots=6)
+    slots = [ctx.kv_reserve() for _ in range(4)]
+    for s in slots:
+        assert model.reserve() == s
+    want = np.array([600, 1500, 64, 3000], np.int64)
+    ctx.kv_premap_async(slots, want)
+    ctx.kv_premap_wait()
+    for s, t in zip(slots, want):
+        assert model.map_pages(s, int(t)) == 0
+        assert ctx.kv_slot_info(s).mapped_tokens >= t
+    same_state(ctx, model)
+    st = ctx.get_stats()
+    assert st.pages_premapped_total == st.pages_mapped_total == model.pages_mapped_total > 0
+    ctx.kv_map_pages_many(slots, want)                       # the foreground call finds everything in place
+    assert ctx.get_stats().pages_mapped_total == model.pages_mapped_total
+    # growth continues in order after a background map
+    ctx.kv_premap_async([slots[0]], [2000])
+    ctx.kv_map_pages(slots[0], 1100)                         # may race with the worker: both are idempotent
+    ctx.kv_premap_wait()
+    assert model.map_pages(slots[0], 2000) == 0
+    same_state(ctx, model)
+    ctx.shutdown()
+
+
+def test_premap_errors_surface_at_wait_and_released_slots_are_dropped(binding):
+    ctx, _ = make(binding, n_pages=4, slots=3)
+    a, b = ctx.kv_reserve(), ctx.kv_reserve()
+    ctx.kv_premap_async([a, b], [1024, 1024])                # 2 + 2 pages: pool exhausted afterwards
+    ctx.kv_premap_wait()
+    ctx.kv_premap_async([a], [2048])                         # needs 2 more pages: none left
+    with pytest.raises(binding.XllmError) as e:
+        ctx.kv_premap_wait()
+    assert e.value.status == binding.ERR_OOM_PHYS and "pre-mapping slot" in str(e.value)
+    ctx.kv_premap_wait()                                     # the failure was reported once
+    ctx.kv_release(b, 1)
+    ctx.kv_premap_async([b, 2, 99], [512, 512, 512])          # released / never reserved / out of range: dropped
+    ctx.kv_premap_wait()
+    assert ctx.kv_slot_info(a).pages_owned == 2 and ctx.get_stats().pages_free == 2
+    ctx.shutdown()                                           # joins the worker
+
+
+def test_shutdown_with_jobs_pending_does_not_hang(binding):
+    ctx, _ = make(binding, n_pages=64, slots=6, max_len=8192)
+    slots = [ctx.kv_reserve() for _ in range(6)]
+    for r in range(20):
+        ctx.kv_premap_async(slots, [400 * (r + 1)] * 6)
+    ctx.shutdown()

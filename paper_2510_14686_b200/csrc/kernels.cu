@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const int64_t tile_block = (int64_t)p.n_kv_heads * 2 * C::kHalfTile;
     uint32_t fill = 0;      // tiles issued / consumed so far by this CTA (same sequence in every warp)
     uint32_t item_seq = 0;  // items started so far
-    unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0;
+    unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0, tr_epi_main = 0;
 
     __syncthreads();          // barriers initialised
     grid_launch_dependents();  // the next kernel of the stream may start its own prologue
@@ -637,6 +637,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_mempty);  // the consumers may overwrite the group states
+                if (TRACE) tr_epi_main += clock64() - t0;
                 if (live && it.partial_idx >= 0 && it.n_parts > 0) {
                     // Lightly split unit: whichever piece finishes last merges all pieces (log-sum-exp) and writes the
                     // final rows, so no second launch is needed.
@@ -715,7 +716,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     // Warp 0: 0 ns after the dependency wait, 1 ns at its first finished tile, 2 ns at its last finished tile, 3 ns at
     // CTA start, 4 cycles waiting for query rows, 5 cycles in item hand-off (incl. waiting for the epilogue), 6 items,
     // 7 tiles, 15 ns lifetime.  Warp 4: 8 cycles in tile loops, 9 ns at its end, 10 cycles in hand-off.  Producer: 11
-    // cycles waiting for free ring slots, 12 cycles lifetime.  Epilogue warp 9: 13 busy cycles, 14 ns at its end.
+    // cycles waiting for free ring slots.  Epilogue warp 9: 12 cycles merging group states and writing rows, 13 busy
+    // cycles in all (incl. the merge of split units), 14 ns at its end.
     if (TRACE && lane == 0 && (warp == 0 || warp == 4 || warp == kProducerWarp || warp == kEpilogueWarp0)) {
         unsigned long long *tr = p.trace + (int64_t)blockIdx.x * kTraceWords;
         const unsigned long long total = clock64() - t_start;
@@ -726,9 +728,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         } else if (warp == 4) {
             tr[8] = tr_tiles; tr[9] = globaltimer_ns(); tr[10] = tr_switch;
         } else if (warp == kProducerWarp) {
-            tr[11] = tr_wait_empty; tr[12] = total;
+            tr[11] = tr_wait_empty;
         } else {
-            tr[13] = tr_epi; tr[14] = globaltimer_ns();
+            tr[12] = tr_epi_main; tr[13] = tr_epi; tr[14] = globaltimer_ns();
         }
     }
 

@@ -337,13 +337,26 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     value = job_throughput(tokens_per_step, world, args.steps, ms)
     e2e_value = job_throughput(tokens_per_step, world, args.steps, ms_e2e)
+    # Duration of the dominant kernel.  Two live measurements: (a) CUDA events recorded by the library right around
+    # each attention launch in a second pass over the same steps -- for a ~50 us kernel the two event records and the
+    # lost launch overlap add several us; (b) when a step launches exactly one kernel (the fused append + attention
+    # call), the events around the K timed steps divided by K: the kernel's average launch-to-launch time, an upper
+    # bound on its duration that still contains the host-side gaps.  The smaller of the two is reported; both are given.
+    attn_ms_bracketed = attn_ms
+    one_kernel_per_step = launches == args.steps
+    if one_kernel_per_step and 0 < ms / args.steps < attn_ms:
+        attn_ms = ms / args.steps
     achieved = alg_bytes / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
     h2d = int(rep.h_q.numel() + rep.h_k.numel() + rep.h_v.numel()) * 2
     d2h = int(rep.h_out.numel()) * 2
 
     # CPU baseline: the oracle, untouched, on this machine's host cores, on a bounded sample of the same workload
-    sample = oracle_sample(name, sample_size(name))
+    # (about 10-30 s of CPU work: passes over the sample are repeated until ~1.5 s of wall clock on all cores)
+    sample = oracle_sample(name, 4 * sample_size(name))
     cpu_tps, cpu_dt, cores = time_oracle(sample, 1)
+    cpu_passes = int(max(1, min(50, 1.5 / max(cpu_dt, 1e-3))))
+    if cpu_passes > 1:
+        cpu_tps, cpu_dt, cores = time_oracle(sample, cpu_passes)
 
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
@@ -360,10 +373,13 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "kernel": "attention_kernel (split-KV)",
                      "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": attn_ms,
+                     "kernel_ms_event_bracketed": attn_ms_bracketed,
+                     "kernel_ms_source": ("timed region / steps (one kernel per step)" if attn_ms != attn_ms_bracketed
+                                          else "events around each launch"),
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "combine_kernel_ms": comb_ms, "append_kernel_ms": app_ms},
         "cpu_baseline": {"value": cpu_tps, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"first {len(sample.requests)} of {s.batch} requests ({sample.kv_tokens} KV tokens), 1 pass, {cpu_dt:.2f} s"},
+                         "sample": f"first {len(sample.requests)} of {s.batch} requests ({sample.kv_tokens} KV tokens), {cpu_passes} passes of {cpu_dt:.2f} s on {cores} threads"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": launches, "clocks": clocks,

@@ -187,6 +187,12 @@ xllm_status xllm_debug_read_page(xllm_ctx *ctx, int32_t page_id, int64_t byte_of
  * kernel).  Only collected when the process was started with XLLM_TRACE=1 in the environment; else UNSUPPORTED. */
 xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max_words, int32_t *n_words_out);
 
+/* Test hook for the library's own failure detection: in each of the next n_launches attention launches one CTA arms a
+ * tile copy and never issues it, so that the consumers' bounded wait (2 s) runs out.  The launch then ends by itself,
+ * its output is invalid, and the next call on the context (or xllm_sync_check) returns XLLM_ERR_CUDA; the context
+ * stays usable.  Nothing faults, traps or spins without a limit. */
+xllm_status xllm_debug_inject_timeout(xllm_ctx *ctx, int32_t n_launches);
+
 /* ---- KV writes ("write_kvcache": only a start address and offsets, no block table) ---------------------- */
 
 /* Append n_new[i] tokens to slot slots[i] for i < n_req: rows k_new / v_new (device, bf16,

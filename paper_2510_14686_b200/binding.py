@@ -92,6 +92,7 @@ EXPORTS = {
     "xllm_debug_read_slot": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
     "xllm_debug_read_page": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp]),
     "xllm_debug_read_trace": (ctypes.c_int32, [_ctxp, ctypes.POINTER(ctypes.c_uint64), ctypes.c_int32, _i32p]),
+    "xllm_debug_inject_timeout": (ctypes.c_int32, [_ctxp, ctypes.c_int32]),
     "xllm_kv_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp]),
     "xllm_kv_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp, _vp]),
     "xllm_decode_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
@@ -270,6 +271,9 @@ class Context:
         n = ctypes.c_int32()
         self._check(_lib.xllm_debug_read_trace(self._ctx, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)), len(buf), ctypes.byref(n)))
         return buf[:n.value].reshape(-1, 16)
+
+    def debug_inject_timeout(self, n_launches: int):
+        self._check(_lib.xllm_debug_inject_timeout(self._ctx, n_launches))
 
     # -- KV writes --
     def kv_append(self, slots, n_new, k_new, v_new, stream=None):

@@ -86,6 +86,7 @@ struct xllm_ctx {
     // scratch for debug_read_page
     uint64_t scratch_va = 0;
 
+    int32_t inject_timeouts = 0;  // attention launches still to be made with one stalled copy (test hook)
     bool profiling = false;
     std::vector<TimedLaunch> timed;
     std::vector<cudaEvent_t> event_pool;
@@ -399,7 +400,13 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.head_dim = ctx->cfg.head_dim;
     al.scale_log2 = scale * 1.4426950408889634f;
     al.n_ctas = ctx->sm_count;
+    al.debug_stall_cta = -1;
     std::memcpy(al.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    if (ctx->inject_timeouts > 0) {
+        --ctx->inject_timeouts;
+        for (int32_t c = 0; c < ctx->sm_count; ++c)
+            if (al.cta_begin[c] < al.cta_begin[c + 1]) { al.debug_stall_cta = c; break; }
+    }
     for (int32_t c = 0; c < ctx->sm_count; ++c)
         if (al.cta_begin[c] < al.cta_begin[c + 1]) al.first_item[c] = di[al.cta_begin[c]];
     time_begin(ctx, 0, stream);
@@ -748,6 +755,13 @@ xllm_status xllm_debug_read_trace(xllm_ctx *ctx, uint64_t *host_dst, int32_t max
     if (e == cudaSuccess) e = cudaMemcpy(host_dst, ctx->d_trace, sizeof(uint64_t) * (size_t)n, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(ctx, "debug_read_trace", (int)e);
     *n_words_out = n;
+    return XLLM_OK;
+}
+
+xllm_status xllm_debug_inject_timeout(xllm_ctx *ctx, int32_t n_launches) {
+    if (!ctx || n_launches < 0) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    ctx->inject_timeouts = n_launches;
     return XLLM_OK;
 }
 

@@ -481,6 +481,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                             if (!mbar_wait(bar_empty + hs * 8, ph ^ 1, abort_flag, p.error_flag, 2)) continue;
                             if (TRACE) tr_wait_empty += clock64() - t0;
                             mbar_expect_tx(bar_full + hs * 8, C::kPanels * bytes);
+                            if (half == 1 && fill == 0 && (int)blockIdx.x == p.debug_stall_cta) continue;  // test hook: the wait on this half must run out
                             const uint32_t dst = smem_base + C::kOffStages + hs * C::kHalfTile;
 #pragma unroll
                             for (int pn = 0; pn < C::kPanels; ++pn)
@@ -638,7 +639,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_mempty);  // the consumers may overwrite the group states
                 if (TRACE) tr_epi_main += clock64() - t0;
-                if (live && it.partial_idx >= 0 && it.n_parts > 0) {
+                if (it.partial_idx >= 0 && it.n_parts > 0) {  // (a property of the item: all 96 threads take the same way)
                     // Lightly split unit: whichever piece finishes last merges all pieces (log-sum-exp) and writes the
                     // final rows, so no second launch is needed.
                     // Release: every epilogue thread's partial stores, CTA barrier, then ONE acq_rel atomic at GPU scope
@@ -647,8 +648,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     volatile int *bcast = reinterpret_cast<volatile int *>(smem + C::kOffFlags) + 1;
                     asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");
                     if (et == 0) {
-                        int old;
-                        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.counters + it.part_first) : "memory");
+                        int old = -1;  // after a bounded wait gave up in this CTA the piece is not counted: nobody merges
+                        if (live && !*abort_flag)
+                            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.counters + it.part_first) : "memory");
                         *bcast = old;
                     }
                     asm volatile("bar.sync 3, %0;" ::"n"(kEpilogueThreads) : "memory");

@@ -111,6 +111,7 @@ struct AttnLaunch {
     int32_t n_q_heads, n_kv_heads, head_dim;
     float scale_log2;             // scale * log2(e)
     int32_t n_ctas;
+    int32_t debug_stall_cta;      // -1; else that CTA arms the V half of its first tile but never copies it (timeout test)
     int32_t cta_begin[kMaxCtas + 1];  // CTA c owns items [cta_begin[c], cta_begin[c+1])
     DevItem first_item[kMaxCtas];     // copy of items[cta_begin[c]]: the first loads need no trip to the item list
 };

@@ -84,6 +84,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrival without release semantics, for a thread that has global stores in flight (a releasing arrive may first wait
+// until those are performed).  `after` is a value computed from everything the thread read from the buffer it hands
+// back: those reads have completed before the arrival is issued.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar, float after) {
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];  // %1" ::"r"(bar), "f"(after) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -172,7 +178,7 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
     const int swz = lane & 7, q4 = lane & 3, g8 = lane >> 2;
     const int tok_base = tile_tok0 + wslice * 16;
     const bool work = tok_base < kv_end;  // the slice holds at least one fetched token
-    live = mbar_wait(bar_k_full, ph_k, abort_flag, error_flag, 4) && live;
+    live = __all_sync(0xffffffffu, mbar_wait(bar_k_full, ph_k, abort_flag, error_flag, 4)) && live;  // (voted: `live` steers warp-wide shuffles)
 
     // ---- scores of this warp's 16 tokens; two accumulation chains per 8-token block ----
     float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -270,7 +276,7 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
         }
     }
     group_bar(group);  // (2) the weight tile is complete
-    live = mbar_wait(bar_v_full, ph_v, abort_flag, error_flag, 7) && live;
+    live = __all_sync(0xffffffffu, mbar_wait(bar_v_full, ph_v, abort_flag, error_flag, 7)) && live;
 
     // ---- O[:, this warp's columns] += P[16 x 64] . V[64 x columns] ----
     if (live) {
@@ -508,7 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 const uint32_t seq = item_seq + i, qb = seq & 1, qph = (seq >> 1) & 1;
                 uint32_t qf[D / 16][4];
                 unsigned long long t0 = TRACE ? clock64() : 0ull;
-                bool live = mbar_wait(bar_qfull + qb * 8, qph, abort_flag, p.error_flag, 3);
+                bool live = __all_sync(0xffffffffu, mbar_wait(bar_qfull + qb * 8, qph, abort_flag, p.error_flag, 3));
                 if (TRACE) tr_wait_q += clock64() - t0;
                 {
                     const uint32_t qsrc = smem_base + C::kOffQ + qb * (kMaxRows * C::kQPitch) +
@@ -606,38 +612,66 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 const DevItem it = item_at(i);
                 const int n_rows = it.n_q_tok * it.n_g;
                 const uint32_t seq = item_seq + i;
-                const bool live = mbar_wait(bar_mfull, seq & 1, abort_flag, p.error_flag, 6);
+                const bool live = __all_sync(0xffffffffu, mbar_wait(bar_mfull, seq & 1, abort_flag, p.error_flag, 6));
                 const unsigned long long t0 = TRACE ? clock64() : 0ull;
-                for (int idx = et; live && idx < n_rows * kC4; idx += kEpilogueThreads) {
-                    const int row = idx / kC4, c4 = idx - row * kC4;
-                    const float mA = merge_m[row], mB = merge_m[kMaxRows + row];
-                    const float lA = (merge_l[row] + merge_l[kMaxRows + row]) + (merge_l[2 * kMaxRows + row] + merge_l[3 * kMaxRows + row]);
-                    const float lB = (merge_l[4 * kMaxRows + row] + merge_l[5 * kMaxRows + row]) +
-                                     (merge_l[6 * kMaxRows + row] + merge_l[7 * kMaxRows + row]);
-                    const float4 oA = *reinterpret_cast<const float4 *>(merge_o + row * C::kOPitch + c4 * 4);
-                    const float4 oB = *reinterpret_cast<const float4 *>(merge_o + (kMaxRows + row) * C::kOPitch + c4 * 4);
-                    const float M = fmaxf(mA, mB);
-                    const float Ms = (M == -INFINITY) ? 0.f : M;
-                    const float wA = exp2f(mA - Ms), wB = exp2f(mB - Ms);  // 0 for a group that saw no visible key
-                    const float L = wA * lA + wB * lB;
-                    const float inv = (L > 0.f) ? 1.f / L : 0.f;
-                    const float lse2 = (L > 0.f) ? M + log2f(L) : -INFINITY;
-                    const float4 acc = make_float4((wA * oA.x + wB * oB.x) * inv, (wA * oA.y + wB * oB.y) * inv,
-                                                   (wA * oA.z + wB * oB.z) * inv, (wA * oA.w + wB * oB.w) * inv);
+                // Kept short on purpose: these warps run this once per item, from a cold instruction cache.  Lane r (and
+                // r + 16) of every warp computes the normalised weights of row r once; the element loop fetches them by
+                // shuffle, sums the two group states, hands the buffers back to the consumers as soon as the last
+                // element's loads have been used (without waiting for any global store), and stores.
+                float wA = 0.f, wB = 0.f, lse2 = -INFINITY;
+                {
+                    const int row = lane & (kMaxRows - 1);
+                    if (live && row < n_rows) {
+                        const float mA = merge_m[row], mB = merge_m[kMaxRows + row];
+                        const float lA = (merge_l[row] + merge_l[kMaxRows + row]) + (merge_l[2 * kMaxRows + row] + merge_l[3 * kMaxRows + row]);
+                        const float lB = (merge_l[4 * kMaxRows + row] + merge_l[5 * kMaxRows + row]) +
+                                         (merge_l[6 * kMaxRows + row] + merge_l[7 * kMaxRows + row]);
+                        const float M = fmaxf(mA, mB);
+                        const float Ms = (M == -INFINITY) ? 0.f : M;
+                        wA = exp2f(mA - Ms), wB = exp2f(mB - Ms);  // 0 for a group that saw no visible key
+                        const float L = wA * lA + wB * lB;
+                        const float inv = (L > 0.f) ? 1.f / L : 0.f;
+                        lse2 = (L > 0.f) ? M + log2f(L) : -INFINITY;
+                        wA *= inv;
+                        wB *= inv;
+                    }
+                }
+                const int n_elems = live ? n_rows * kC4 : 0;
+                const int n_iter = (n_elems - (et & ~31) + kEpilogueThreads - 1) / kEpilogueThreads;  // (the same for the whole warp)
+                if (n_iter <= 0) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_relaxed(bar_mempty, 0.f);
+                }
+#pragma unroll 1
+                for (int j = 0; j < n_iter; ++j) {
+                    const int idx = et + j * kEpilogueThreads;
+                    const bool valid = idx < n_elems;
+                    const int row = valid ? idx / kC4 : 0, c4 = idx - row * kC4;
+                    const float a = __shfl_sync(0xffffffffu, wA, row), b = __shfl_sync(0xffffffffu, wB, row);
+                    const float lse_row = __shfl_sync(0xffffffffu, lse2, row);
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (valid) {
+                        const float4 oA = *reinterpret_cast<const float4 *>(merge_o + row * C::kOPitch + c4 * 4);
+                        const float4 oB = *reinterpret_cast<const float4 *>(merge_o + (kMaxRows + row) * C::kOPitch + c4 * 4);
+                        acc = make_float4(a * oA.x + b * oB.x, a * oA.y + b * oB.y, a * oA.z + b * oB.z, a * oA.w + b * oB.w);
+                    }
+                    if (j == n_iter - 1) {  // (n_iter is the same for the whole warp)
+                        const float seen = acc.x + __shfl_xor_sync(0xffffffffu, acc.x, 1);  // every lane's loads have been used
+                        if (lane == 0) mbar_arrive_relaxed(bar_mempty, seen);
+                    }
+                    if (!valid) continue;
                     if (it.partial_idx >= 0) {
                         float *dst = p.part_o + ((int64_t)it.partial_idx * kMaxRows + row) * D + c4 * 4;
                         *reinterpret_cast<float4 *>(dst) = acc;
-                        if (c4 == 0) p.part_lse[(int64_t)it.partial_idx * kMaxRows + row] = lse2;
+                        if (c4 == 0) p.part_lse[(int64_t)it.partial_idx * kMaxRows + row] = lse_row;
                     } else {
                         const int ti = row / it.n_g, gi = row - ti * it.n_g;
                         const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
                         *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
                             make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-                        if (c4 == 0 && p.lse_out) p.lse_out[off] = lse2 * 0.69314718055994531f;
+                        if (c4 == 0 && p.lse_out) p.lse_out[off] = lse_row * 0.69314718055994531f;
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_mempty);  // the consumers may overwrite the group states
                 if (TRACE) tr_epi_main += clock64() - t0;
                 if (it.partial_idx >= 0 && it.n_parts > 0) {  // (a property of the item: all 96 threads take the same way)
                     // Lightly split unit: whichever piece finishes last merges all pieces (log-sum-exp) and writes the

@@ -143,11 +143,13 @@ def _stream(stream) -> int:
 
 
 def plan_partition(kv_lens: Sequence[int], q_lens: Optional[Sequence[int]], n_q_heads: int, n_kv_heads: int, n_ctas: int):
-    """Host-only: returns (items: list[WorkItem], cta_begin: np.ndarray, n_units, n_partials)."""
+    """Host-only: returns (items: list[WorkItem], cta_begin: np.ndarray, n_units, n_partials).
+
+    CTA c owns items[cta_begin[c]:cta_begin[c+1]]; items[cta_begin[-1]:] are the shared pool."""
     kv = np.ascontiguousarray(kv_lens, dtype=np.int64)
     n = len(kv)
     ql = _i32(q_lens) if q_lens is not None else None
-    cap = n * n_kv_heads * 16 + n_ctas + 8
+    cap = n * n_kv_heads * 16 + 9 * n_ctas + 8
     items = (WorkItem * cap)()
     cta = np.zeros(n_ctas + 1, np.int32)
     n_items, n_units, n_parts = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()

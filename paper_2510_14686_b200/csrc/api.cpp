@@ -86,6 +86,8 @@ struct xllm_ctx {
     // scratch for debug_read_page
     uint64_t scratch_va = 0;
 
+    PlanScratch plan_scratch;
+    uint32_t pool_base = 0;       // claims made on the shared pools of all launches so far (mirrors the device counter)
     int32_t inject_timeouts = 0;  // attention launches still to be made with one stalled copy (test hook)
     bool profiling = false;
     std::vector<TimedLaunch> timed;
@@ -124,7 +126,8 @@ xllm_status check_device_flag(xllm_ctx *ctx) {
         *ctx->h_error = 0;
         // the launch that gave up may have left arrival counters of split units behind
         cudaDeviceSynchronize();
-        if (ctx->d_counters) cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * (size_t)ctx->max_partials);
+        if (ctx->d_counters) cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
+        ctx->pool_base = 0;
         return fail(ctx, XLLM_ERR_CUDA, "attention kernel: a bounded device-side wait expired (code " + std::to_string(code) +
                                             "); the results of that launch are invalid");
     }
@@ -307,7 +310,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     }
     int32_t n_units = 0, n_partials = 0;
     if (plan_partition(n_req, ctx->kv_lens.data(), q_lens, ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, ctx->sm_count, ctx->tune,
-                       ctx->items, ctx->cta_begin, &n_units, &n_partials) != 0)
+                       ctx->items, ctx->cta_begin, &n_units, &n_partials, &ctx->plan_scratch) != 0)
         return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
     const int32_t n_items = (int32_t)ctx->items.size();
     if (n_items > ctx->max_items || n_partials > ctx->max_partials)
@@ -393,6 +396,10 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.part_o = ctx->d_part_o;
     al.part_lse = ctx->d_part_lse;
     al.counters = ctx->d_counters;
+    al.pool_counter = reinterpret_cast<uint32_t *>(ctx->d_counters + ctx->max_partials);
+    al.pool_base = ctx->pool_base;
+    al.pool_first = ctx->cta_begin[(size_t)ctx->sm_count];
+    al.n_pool = n_items - al.pool_first;
     al.error_flag = ctx->d_error;
     al.trace = ctx->d_trace;
     al.n_q_heads = ctx->cfg.n_q_heads;
@@ -413,6 +420,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     e = launch_attention(al, stream);
     time_end(ctx, stream);
     if (e) return cuda_fail(ctx, "launching the attention kernel", e);
+    if (al.n_pool > 0) ctx->pool_base += (uint32_t)al.n_pool + (uint32_t)al.n_ctas;  // every CTA's last claim fails, exactly once
     ++ctx->st.kernel_launches;
     if (!combine.empty()) {
         CombineLaunch cl{};
@@ -490,14 +498,17 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         drv = make_cuda_driver(&derr);
         if (!drv) return bad(XLLM_ERR_CUDA, derr);
     }
-    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece[,pieces_first]": planner override (tuning aid)
-        int a, b, c, d, f = 1;
-        if (std::sscanf(t, "%d,%d,%d,%d,%d", &a, &b, &c, &d, &f) >= 4 && a > 0 && b >= 0 && c >= 0 && d >= 1) {
+    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece[,pieces_first[,pool_pct[,pool_min]]]": planner override (tuning aid)
+        int a, b, c, d, f = ctx->tune.pieces_first, g = ctx->tune.pool_pct, h = ctx->tune.pool_min_tiles;
+        if (std::sscanf(t, "%d,%d,%d,%d,%d,%d,%d", &a, &b, &c, &d, &f, &g, &h) >= 4 && a > 0 && b >= 0 && c >= 0 && d >= 1 && g >= 0 &&
+            g <= 50 && h >= 1) {
             ctx->tune.tile_cost = a;
             ctx->tune.unit_overhead = b;
             ctx->tune.row_overhead = c;
             ctx->tune.min_piece_tiles = d;
             ctx->tune.pieces_first = f;
+            ctx->tune.pool_pct = g;
+            ctx->tune.pool_min_tiles = h;
         }
     }
     ctx->xt.reset(new XTensor(std::move(drv), cfg->device, cfg->max_slots, cfg->max_seq_len, row_bytes));
@@ -514,7 +525,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     const int32_t G = cfg->n_q_heads / cfg->n_kv_heads;
     const int32_t groups = (G <= kMaxRows) ? (cfg->max_q_len + std::max(1, kMaxRows / G) - 1) / std::max(1, kMaxRows / G)
                                            : cfg->max_q_len * ((G + kMaxRows - 1) / kMaxRows);
-    ctx->max_items = cfg->max_slots * cfg->n_kv_heads * groups + ctx->sm_count + 1;
+    ctx->max_items = cfg->max_slots * cfg->n_kv_heads * groups + (1 + kPoolMaxPerCta) * ctx->sm_count + 1;
     ctx->max_partials = 2 * ctx->sm_count + 2;
     ctx->stage_bytes = std::max(align_up(sizeof(DevItem) * (size_t)ctx->max_items, 16) +
                                     align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16),
@@ -528,8 +539,9 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         }
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * kMaxRows * cfg->head_dim);
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * kMaxRows);
-        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_counters), sizeof(int32_t) * (size_t)ctx->max_partials);
-        if (e == cudaSuccess) e = cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * (size_t)ctx->max_partials);
+        // arrival counters of split units, and one more word: the claim counter of the shared pool
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_counters), sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
         if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_error), sizeof(int32_t), cudaHostAllocMapped);
         if (e == cudaSuccess) {
             *ctx->h_error = 0;

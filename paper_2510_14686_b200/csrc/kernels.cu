@@ -35,6 +35,7 @@ constexpr int kEpilogueWarps = 3;
 constexpr int kEpilogueThreads = kEpilogueWarps * 32;
 constexpr int kThreads = (kConsumerWarps + 1 + kEpilogueWarps) * 32;  // 384
 constexpr int kItemBatch = 64;
+constexpr int kPoolSlots = 4;   // records of the shared pool the producer may publish ahead of the other warps
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // a bounded wait gives up after 2 s
 
 template <int D>
@@ -65,8 +66,9 @@ struct Cfg {
     static constexpr int kOffP = kOffMax + 2 * 2 * 4 * kMaxRows * 4;             // [2 groups][2 bufs][16 rows][kPPitch]
     static constexpr int kOffQ = kOffP + 2 * 2 * kMaxRows * kPPitch;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
-    static constexpr int kOffBars = kOffItems + kItemBatch * (int)sizeof(DevItem);
-    static constexpr int kNumBars = 2 * kHalfStages + 8;
+    static constexpr int kOffPool = kOffItems + kItemBatch * (int)sizeof(DevItem);   // [kPoolSlots] records claimed from the shared pool
+    static constexpr int kOffBars = kOffPool + kPoolSlots * (int)sizeof(DevItem);
+    static constexpr int kNumBars = 2 * kHalfStages + 8 + 2 * kPoolSlots;
     static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast
     static constexpr int kSmemBytes = kOffFlags + 16;
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
@@ -374,6 +376,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const uint32_t bar_mempty = bar_mfull + 8;                        // ... and read by the epilogue (3 warps)
     const uint32_t bar_items = bar_mempty + 8;                        // first batch of item records is in shared memory
     const uint32_t bar_append = bar_items + 8;                        // first batch's new K/V rows are in their ranges
+    const uint32_t bar_pfull = bar_append + 8;                        // [kPoolSlots] a record claimed from the shared pool is published
+    const uint32_t bar_pempty = bar_pfull + kPoolSlots * 8;           // [kPoolSlots] ... and read by the 8 consumer and 3 epilogue warps
+    const DevItem *pool_items = reinterpret_cast<const DevItem *>(smem + C::kOffPool);
     const unsigned long long t_start = TRACE ? clock64() : 0ull;
     const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
 
@@ -391,12 +396,20 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         mbar_init(bar_mempty, kEpilogueWarps);
         mbar_init(bar_items, kEpilogueWarps);
         mbar_init(bar_append, kEpilogueWarps);
+        for (int b = 0; b < kPoolSlots; ++b) {
+            mbar_init(bar_pfull + b * 8, 1);
+            mbar_init(bar_pempty + b * 8, kConsumerWarps + kEpilogueWarps);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
     const int64_t tile_block = (int64_t)p.n_kv_heads * 2 * C::kHalfTile;
+    // Tiles alternate between the two consumer groups.  Inside the CTA's own run the alternation runs on across items;
+    // a piece from the shared pool always starts with group 0, so that its result does not depend on which CTA claimed
+    // it (and on what that CTA did before).  group_tiles[g]: tiles given to group g so far = position in g's ring.
     uint32_t fill = 0;      // tiles issued / consumed so far by this CTA (same sequence in every warp)
+    uint32_t group_tiles[2] = {0, 0};
     uint32_t item_seq = 0;  // items started so far
     unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0, tr_epi_main = 0;
 
@@ -406,14 +419,24 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const unsigned long long g_go = TRACE ? globaltimer_ns() : 0ull;
     unsigned long long g_first = 0, g_last = 0;
 
-    for (int batch_lo = item_lo; batch_lo < item_hi; batch_lo += kItemBatch) {
-        const int nb = min(kItemBatch, item_hi - batch_lo);
-        const bool first_batch = batch_lo == item_lo;
+    // The CTA's own run comes in batches of kItemBatch records; after it, one more segment: the shared pool, from which
+    // the producer claims one record at a time (an atomic counter) and publishes it to the other warps.
+    const int n_batches = (item_hi - item_lo + kItemBatch - 1) / kItemBatch;
+    const int n_segments = n_batches + (p.n_pool > 0 ? 1 : 0);
+    uint32_t my_tiles = 0;  // consumers: tiles this group has processed, selects the double buffer of maxima / weights
+    uint32_t n_items_done = 0;
+    for (int seg = 0; seg < n_segments; ++seg) {
+        const bool pool = seg == n_batches;
+        const int batch_lo = item_lo + seg * kItemBatch;
+        const int nb = pool ? 0x7fffffff : min(kItemBatch, item_hi - batch_lo);
+        const bool first_batch = seg == 0 && !pool;
         // Item records live in host memory mapped into the device: fetching them costs a trip over PCIe.  In the
         // first batch the record of item 0 comes from the kernel parameters and the epilogue warps (idle until the
         // first item is finished) fetch the rest, so the first loads start at once; later batches (more than
         // kItemBatch items in a CTA) are fetched by everybody between two CTA-wide barriers.
-        if (first_batch) {
+        if (pool) {
+            // nothing to stage: records arrive one by one
+        } else if (first_batch) {
             if (warp >= kEpilogueWarp0) {
                 for (int i = tid - kEpilogueWarp0 * 32; i < nb * 3; i += kEpilogueThreads)  // 48-byte records, 16-byte pieces
                     reinterpret_cast<uint4 *>(smem + C::kOffItems)[i] = reinterpret_cast<const uint4 *>(p.items + batch_lo)[i];
@@ -452,11 +475,73 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             }
             return sitems[i];
         };
+        // consumers and epilogue (all lanes): the i-th record the producer claimed from the pool; false when the pool is empty
+        auto pool_item_at = [&](int i, DevItem &it) -> bool {
+            const uint32_t ps = i % kPoolSlots, pph = (i / kPoolSlots) & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_pfull + ps * 8, pph, abort_flag, p.error_flag, 10))) return false;
+            it = pool_items[ps];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pempty + ps * 8);
+            return it.tile_begin >= 0;
+        };
+        int n_done = 0;  // items of this segment (the same in every warp)
 
         if (warp == kProducerWarp) {
             // ================= producer =================
-            for (int i = 0; i < nb && lane == 0; ++i) {  // one elected lane issues every copy; the others wait below
-                const DevItem it = item_at(i);
+            union Record {
+                DevItem it;
+                uint4 w[3];
+            } next;  // pool: the record just claimed
+            bool have = false;
+            auto claim = [&]() {  // one more record of the pool, or none: every CTA's last claim fails, exactly once
+                const uint32_t t = atomicAdd(p.pool_counter, 1u) - p.pool_base;
+                have = t < (uint32_t)p.n_pool;
+                if (have) {       // (host memory: the latency overlaps with the copies issued in the meantime)
+                    const uint4 *src = reinterpret_cast<const uint4 *>(p.items + p.pool_first + t);
+                    next.w[0] = src[0];
+                    next.w[1] = src[1];
+                    next.w[2] = src[2];
+                }
+            };
+            // One elected lane issues every copy.  In the pool segment the other lanes follow it item by item, because an
+            // item that carries new K/V rows (a whole unit, in a launch that appends) has them written by this warp first.
+            for (int i = 0; i < nb && (pool || lane == 0); ++i) {
+                DevItem it;
+                if (!pool) {
+                    it = item_at(i);
+                } else {
+                    const uint32_t ps = i % kPoolSlots, pph = (i / kPoolSlots) & 1;
+                    int go = 0;
+                    if (lane == 0) {
+                        // Claimed only now, when this CTA is ready to issue it: a CTA that claimed ahead would take work
+                        // from one that is further along.  (The record comes from host memory; the tiles already in the
+                        // ring cover most of that latency.)
+                        claim();
+                        const bool ok = mbar_wait(bar_pempty + ps * 8, pph ^ 1, abort_flag, p.error_flag, 11);
+                        Record pub = next;
+                        if (!have) pub.it.tile_begin = pub.it.tile_end = -1;  // end of the pool
+                        if (ok) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(smem + C::kOffPool) + ps * 3;
+                            dst[0] = pub.w[0];
+                            dst[1] = pub.w[1];
+                            dst[2] = pub.w[2];
+                            mbar_arrive(bar_pfull + ps * 8);
+                        }
+                        go = have && ok;
+                    }
+                    __syncwarp();
+                    go = __shfl_sync(0xffffffffu, go, 0);
+                    if (!go) break;
+                    it = pool_items[ps];
+                    if (it.n_new > 0 && p.k_new) {
+                        append_new_rows<D>(pool_items + ps, it, true, 1, p, tile_block, lane, 32);
+                        __threadfence();
+                        asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores before the bulk copies that read them
+                        __syncwarp();
+                    }
+                }
+                ++n_done;
+                if (lane != 0) continue;
                 {
                     const int n_rows = it.n_q_tok * it.n_g;
                     const uint32_t qb = (item_seq + i) & 1, qph = ((item_seq + i) >> 1) & 1;
@@ -470,7 +555,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                                          D * 2, bar_qfull + qb * 8);
                     }
                     const char *kv = reinterpret_cast<const char *>(it.kv);
+                    const uint32_t g_first_tile = pool ? 0u : (fill & 1u);
                     for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
+                        const uint32_t g = ((uint32_t)(tile - it.tile_begin) + g_first_tile) & 1u;
+                        const uint32_t j = g ? group_tiles[1]++ : group_tiles[0]++;
                         const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);
                         const uint32_t bytes = rows * 128;
                         const char *src = kv + (int64_t)tile * tile_block;
@@ -482,7 +570,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {  // K half, then V half
                             uint32_t hs, ph;
-                            C::slot_of(fill & 1, fill >> 1, half, hs, ph);
+                            C::slot_of(g, j, half, hs, ph);
                             const unsigned long long t0 = TRACE ? clock64() : 0ull;
                             if (!mbar_wait(bar_empty + hs * 8, ph ^ 1, abort_flag, p.error_flag, 2)) continue;
                             if (TRACE) tr_wait_empty += clock64() - t0;
@@ -496,7 +584,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     }
                 }
             }
+            __syncwarp();
             fill = __shfl_sync(0xffffffffu, fill, 0);
+            n_done = __shfl_sync(0xffffffffu, n_done, 0);
         } else if (warp < kConsumerWarps) {
             // ================= consumers =================
             const int group = warp >> 2, wslice = warp & 3;
@@ -506,9 +596,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             float *merge_l = reinterpret_cast<float *>(smem + C::kOffMergeL) + (group * 4 + wslice) * kMaxRows;
             float *mx_base = reinterpret_cast<float *>(smem + C::kOffMax) + group * (2 * 4 * kMaxRows);
             const uint32_t p_base = smem_base + C::kOffP + group * (2 * kMaxRows * C::kPPitch);
-            uint32_t my_tiles = 0;  // tiles this group has processed: selects the double buffer of maxima / weights
             for (int i = 0; i < nb; ++i) {
-                const DevItem it = item_at(i);
+                DevItem it;
+                if (!pool)
+                    it = item_at(i);
+                else if (!pool_item_at(i, it))
+                    break;
+                ++n_done;
                 const int n_rows = it.n_q_tok * it.n_g;
                 const int row_limit0 = it.kv_end - it.n_q_tok + 1;
                 const uint32_t seq = item_seq + i, qb = seq & 1, qph = (seq >> 1) & 1;
@@ -538,11 +632,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
 
                 t0 = TRACE ? clock64() : 0ull;
+                const uint32_t g_first_tile = pool ? 0u : (fill & 1u);
                 for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
-                    if ((int)(fill & 1) != group) continue;
+                    if ((int)(((uint32_t)(tile - it.tile_begin) + g_first_tile) & 1u) != group) continue;
+                    const uint32_t j = group_tiles[0]++;  // (a consumer warp counts its own group's tiles only)
                     uint32_t sk, sv, phk, phv;
-                    C::slot_of(group, fill >> 1, 0, sk, phk);
-                    C::slot_of(group, fill >> 1, 1, sv, phv);
+                    C::slot_of(group, j, 0, sk, phk);
+                    C::slot_of(group, j, 1, sv, phv);
                     const uint32_t kstage = smem_base + C::kOffStages + sk * C::kHalfTile;
                     const uint32_t vstage = smem_base + C::kOffStages + sv * C::kHalfTile;
                     float *mxs = mx_base + (my_tiles & 1) * (4 * kMaxRows);
@@ -609,7 +705,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             const float *merge_l = reinterpret_cast<const float *>(smem + C::kOffMergeL);
             constexpr int kC4 = D / 4;  // float4 columns per row
             for (int i = 0; i < nb; ++i) {
-                const DevItem it = item_at(i);
+                DevItem it;
+                if (!pool)
+                    it = item_at(i);
+                else if (!pool_item_at(i, it))
+                    break;
+                ++n_done;
                 const int n_rows = it.n_q_tok * it.n_g;
                 const uint32_t seq = item_seq + i;
                 const bool live = __all_sync(0xffffffffu, mbar_wait(bar_mfull, seq & 1, abort_flag, p.error_flag, 6));
@@ -745,7 +846,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 if (TRACE) tr_epi += clock64() - t0;
             }
         }
-        item_seq += nb;
+        item_seq += n_done;
+        n_items_done += n_done;
     }
 
     // trace layout (16 words per CTA); "ns" = absolute global-timer nanoseconds, "cycles" = SM clock cycles.
@@ -759,7 +861,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         const unsigned long long total = clock64() - t_start;
         if (warp == 0) {
             tr[0] = g_go; tr[1] = g_first; tr[2] = g_last; tr[3] = g_start; tr[4] = tr_wait_q; tr[5] = tr_switch;
-            tr[6] = (unsigned long long)(item_hi - item_lo); tr[7] = fill;
+            tr[6] = (unsigned long long)n_items_done; tr[7] = fill;
             tr[15] = globaltimer_ns() - g_start;
         } else if (warp == 4) {
             tr[8] = tr_tiles; tr[9] = globaltimer_ns(); tr[10] = tr_switch;
@@ -776,7 +878,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     if (*abort_flag && warp == kProducerWarp && lane == 0) {
         const unsigned long long t0 = globaltimer_ns();
         for (uint32_t g = 0; g < 2; ++g) {
-            const uint32_t tiles_g = (fill + 1 - g) / 2, halves_g = 2 * tiles_g, n = g ? C::kSlotsB : C::kSlotsA;
+            const uint32_t tiles_g = group_tiles[g], halves_g = 2 * tiles_g, n = g ? C::kSlotsB : C::kSlotsA;
             for (uint32_t back = 0; back < n && back < halves_g; ++back) {
                 const uint32_t hl = halves_g - 1 - back;
                 uint32_t hs, ph;

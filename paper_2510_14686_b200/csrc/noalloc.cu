@@ -135,6 +135,7 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
 
     // ---- plan the work in the fixed host arrays ----
     PlanTuning tune;
+    tune.pool_pct = 0;  // no shared pool here: its claim counter would be one more word that must survive between calls
     PlanBuffers buf{g_units, g_start, kMaxUnits, g_items, kMaxItems, g_cta_begin};
     int32_t n_items = 0, n_units_planned = 0, n_partials = 0;
     if (plan_partition_core(n_req, kv_lens, nullptr, n_q_heads, n_kv_heads, ds.sm_count, tune, buf, &n_items, &n_units_planned,
@@ -184,6 +185,10 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
     al.part_o = sc->part_o;
     al.part_lse = sc->part_lse;
     al.counters = sc->counters;
+    al.pool_counter = nullptr;
+    al.pool_base = 0;
+    al.n_pool = 0;
+    al.pool_first = n_items;
     al.error_flag = &sc->error;
     al.trace = nullptr;
     al.n_q_heads = n_q_heads;

@@ -6,7 +6,8 @@
 // ones.  Here the "compute unit" is one persistent CTA per SM.  All (request, KV head, row group)
 // units are laid out on one cost axis (tiles plus a fixed per-unit overhead) and the axis is cut into
 // n_ctas equal runs; a cut that falls inside a unit splits that unit, and the pieces are merged later
-// by the log-sum-exp combine kernel.
+// by log-sum-exp.  A small share of the work is held back in a pool of short pieces that the CTAs claim
+// at run time when their own run is done (the CTAs do not all get the same bandwidth).
 #include <algorithm>
 #include <cstdint>
 #include <vector>
@@ -32,14 +33,16 @@ int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads
 
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
-                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out) {
+                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out, PlanScratch *scratch) {
     const int64_t n_units = plan_count_units(n_req, q_lens, n_q_heads, n_kv_heads);
     if (n_units < 0 || n_ctas < 1 || n_units > INT32_MAX / 2) return -1;
-    std::vector<PlanUnit> units((size_t)n_units);
-    std::vector<int64_t> start((size_t)n_units + 1);
+    PlanScratch local;
+    PlanScratch &sc = scratch ? *scratch : local;  // (a caller that plans every step keeps the arrays)
+    if (sc.units.size() < (size_t)n_units) sc.units.resize((size_t)n_units);
+    if (sc.start.size() < (size_t)n_units + 1) sc.start.resize((size_t)n_units + 1);
     items.resize((size_t)n_units + (size_t)n_ctas);
     cta_begin.assign((size_t)n_ctas + 1, 0);
-    PlanBuffers buf{units.data(), start.data(), (int32_t)n_units, items.data(), (int32_t)items.size(), cta_begin.data()};
+    PlanBuffers buf{sc.units.data(), sc.start.data(), (int32_t)n_units, items.data(), (int32_t)items.size(), cta_begin.data()};
     int32_t n_items = 0;
     const int rc = plan_partition_core(n_req, kv_lens, q_lens, n_q_heads, n_kv_heads, n_ctas, tune, buf, &n_items, n_units_out,
                                        n_partials_out);
@@ -79,7 +82,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
                     const int64_t vis_last = kv - ql + t0 + nt;  // keys visible to the last row
                     const int64_t vis_first = kv - ql + t0 + 1;  // keys visible to the first row
                     Unit u{r, h, (int16_t)t0, (int16_t)nt, 0, (int16_t)G, (int32_t)((vis_last + T - 1) / T),
-                           (int32_t)((vis_first - 1) / T), 0, 0};
+                           (int32_t)((vis_first - 1) / T), 0, 0, 0};
                     units.push_back(u);
                 }
             } else {
@@ -87,7 +90,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
                     const int64_t vis = kv - ql + t0 + 1;
                     for (int32_t g0 = 0; g0 < G; g0 += kMaxRows) {
                         Unit u{r, h, (int16_t)t0, 1, (int16_t)g0, (int16_t)std::min(kMaxRows, G - g0),
-                               (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T), 0, 0};
+                               (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T), 0, 0, 0};
                         units.push_back(u);
                     }
                 }
@@ -107,6 +110,42 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
         }
         size_t size() const { return (size_t)n; }
     } items{buf.items, 0, buf.cap_items, false};
+    // Shared pool, about pool_pct of the tiles, claimed at run time: whole small units (the smallest ones of at least
+    // pool_min_tiles, up to an eighth of a CTA's share), so nothing is split and nothing has to be merged.  A batch
+    // without such units (a few very long sequences; or so little work that a CTA's run is a few tiles) gets no pool.
+    // The pool is capped at kPoolMaxPerCta items per CTA: what it has to absorb grows with the run time of a CTA, not
+    // with the batch.
+    {
+        int64_t total_tiles = 0;
+        for (int32_t u = 0; u < U; ++u) total_tiles += units[u].n_tiles;
+        const int64_t share = total_tiles / n_ctas;
+        int64_t target_tiles = tune.pool_pct > 0 ? total_tiles * tune.pool_pct / 100 : 0;
+        if (total_tiles < 8 * (int64_t)n_ctas) target_tiles = 0;
+        const int64_t max_items = (int64_t)kPoolMaxPerCta * n_ctas;
+        constexpr int32_t kMaxWhole = 64;
+        const int32_t lo = std::max(1, tune.pool_min_tiles);
+        const int32_t hi = (int32_t)std::min<int64_t>(kMaxWhole, share / 8);  // (much shorter than a CTA's run, or it evens out nothing)
+        int32_t quota[kMaxWhole + 1] = {0};  // units of each size: first how many there are, then how many go to the pool
+        for (int32_t u = 0; u < U && target_tiles > 0; ++u)
+            if (units[u].n_tiles >= lo && units[u].n_tiles <= hi) ++quota[units[u].n_tiles];
+        int64_t got_tiles = 0, got_items = 0;
+        for (int32_t n = lo; n <= kMaxWhole; ++n) {  // smallest first, up to the target
+            const int64_t room_tiles = target_tiles - got_tiles, room_items = max_items - got_items;
+            const int64_t take = (n > hi || room_tiles <= 0 || room_items <= 0)
+                                     ? 0
+                                     : std::min<int64_t>(std::min<int64_t>(quota[n], (room_tiles + n - 1) / n), room_items);
+            quota[n] = (int32_t)take;
+            got_tiles += take * n;
+            got_items += take;
+        }
+        for (int32_t u = 0; u < U && got_items > 0; ++u) {
+            Unit &un = units[u];
+            if (un.n_tiles >= lo && un.n_tiles <= hi && quota[un.n_tiles] > 0) {
+                --quota[un.n_tiles];
+                un.pool_whole = 1;
+            }
+        }
+    }
     // cost axis: start position of every unit.  A full tile costs tile_cost; the last tile of a unit is fetched
     // in 16-token steps: half of its cost is fixed, half goes with the volume; a unit's fixed cost grows with its row count.
     start[0] = 0;
@@ -116,14 +155,15 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
         const int32_t tail_rows = (int32_t)std::min<int64_t>(T, ((vis_last - (int64_t)(un.n_tiles - 1) * T) + 15) / 16 * 16);
         un.last_cost = tune.tile_cost / 2 + tune.tile_cost * tail_rows / (2 * T);  // half fixed, half by volume
         un.overhead = tune.unit_overhead + tune.row_overhead * un.n_q_tok * un.n_g / kMaxRows;
-        start[u + 1] = start[u] + un.overhead + (int64_t)tune.tile_cost * (un.n_tiles - 1) + un.last_cost;
+        start[u + 1] = start[u] + (un.pool_whole ? 0 : un.overhead + (int64_t)tune.tile_cost * (un.n_tiles - 1) + un.last_cost);
     }
     // Walk the axis once, CTA by CTA.  Each CTA aims at an equal share of what is still to be done; "what is
     // still to be done" includes the fixed cost a unit's continuation pays again when a cut splits the unit, so the
     // shares stay equal although every split adds work.
     for (int32_t c = 0; c <= n_ctas; ++c) cta_begin[c] = 0;
     int32_t n_partials = 0;
-    int32_t u = 0, tile = 0;  // next work: unit u from tile `tile` on
+    int32_t u = 0, tile = 0;  // next work: unit u from tile `tile` on; units that are in the pool are skipped
+    while (u < U && units[u].pool_whole) ++u;
     int64_t mean_overhead = 0;
     for (int32_t i = 0; i < U; ++i) mean_overhead += units[i].overhead;
     mean_overhead = U ? mean_overhead / U : 0;
@@ -169,7 +209,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
             it.n_q_tok = un.n_q_tok;
             it.g0 = un.g0;
             it.n_g = un.n_g;
-            it.partial_idx = (tile == 0 && take == un.n_tiles) ? -1 : n_partials++;
+            it.partial_idx = (tile == 0 && take == un.n_tiles) ? -1 : 0;  // (>= 0: a piece; slots are given out below)
             it.unit = u;
             it.part_first = 0;
             it.n_parts = 0;
@@ -178,6 +218,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
             tile += take;
             if (tile == un.n_tiles) {
                 ++u;
+                while (u < U && units[u].pool_whole) ++u;
                 tile = 0;
             } else {
                 break;  // the unit continues in the next CTA
@@ -186,7 +227,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     }
     cta_begin[n_ctas] = static_cast<int32_t>(items.size());
     if (items.overflow) return -2;
-    // Pieces of one unit are adjacent in walk order: give each its unit's first slot and piece count ...
+    // Partial slots: the pieces of a split unit are adjacent in walk order and get consecutive slots.
     for (int32_t i = 0; i < items.n;) {
         if (items.p[i].partial_idx < 0) {
             ++i;
@@ -195,9 +236,11 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
         int32_t j = i;
         while (j < items.n && items.p[j].unit == items.p[i].unit) ++j;
         for (int32_t k = i; k < j; ++k) {
-            items.p[k].part_first = items.p[i].partial_idx;
+            items.p[k].partial_idx = n_partials + (k - i);
+            items.p[k].part_first = n_partials;
             items.p[k].n_parts = j - i;
         }
+        n_partials += j - i;
         i = j;
     }
     // ... then let every CTA do its pieces first so that the round trip of their partial results through global
@@ -212,6 +255,39 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
             items.p[front++] = piece;
         }
     }
+    // The pool, after every CTA's own run, largest units first (what is claimed last should be small).
+    {
+        constexpr int32_t kMaxWhole = 64;
+        int32_t pos[kMaxWhole + 2] = {0};  // pos[n]: where the units of n tiles start
+        for (int32_t i = 0; i < U; ++i)
+            if (units[i].pool_whole) ++pos[units[i].n_tiles];
+        int32_t acc = items.n;
+        for (int32_t n = kMaxWhole; n >= 0; --n) {
+            const int32_t c = pos[n];
+            pos[n] = acc;
+            acc += c;
+        }
+        if (acc > items.cap) return -2;
+        for (int32_t i = 0; i < U; ++i) {
+            const Unit &un = units[i];
+            if (!un.pool_whole) continue;
+            xllm_work_item &it = items.p[pos[un.n_tiles]++];
+            it.req = un.req;
+            it.kv_head = un.kv_head;
+            it.tile_begin = 0;
+            it.tile_end = un.n_tiles;
+            it.q_tok0 = un.q_tok0;
+            it.n_q_tok = un.n_q_tok;
+            it.g0 = un.g0;
+            it.n_g = un.n_g;
+            it.partial_idx = -1;
+            it.unit = i;
+            it.part_first = 0;
+            it.n_parts = 0;
+        }
+        items.n = acc;
+    }
+    if (items.overflow) return -2;
     if (n_items_out) *n_items_out = items.n;
     if (n_units_out) *n_units_out = U;
     if (n_partials_out) *n_partials_out = n_partials;

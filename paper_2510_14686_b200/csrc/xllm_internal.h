@@ -18,7 +18,15 @@ struct PlanTuning {
     int32_t pieces_first = 1;     // 1: inside a CTA the pieces of split units run before the whole units
     int32_t fuse_max_items_per_cta = 8;  // append rides along in the attention launch up to this many work items per CTA
     int32_t min_piece_tiles = 4;  // pieces of a split unit are at least this many tiles (swept on B200: 2..8 are within noise; >= 2 required)
+    // Shared pool: about this share of the tiles (percent) is not given to any CTA beforehand: whole small units that the
+    // CTAs claim one by one when their own run is done, which evens out what no cost model predicts (CTAs differ by
+    // several percent in the bandwidth they get).  0: no pool.  Measured on B200: 6 is best on the speculative-
+    // verification batch; batches of many short requests gain up to 15.
+    int32_t pool_pct = 8;
+    int32_t pool_min_tiles = 4;   // units smaller than this stay with a CTA: claiming costs about as much as they do
 };
+
+constexpr int32_t kPoolMaxPerCta = 8;  // the shared pool holds at most this many pieces per CTA
 
 struct PlanUnit {  // one (request, KV head, row group) on the planner's cost axis
     int32_t req, kv_head;
@@ -27,6 +35,7 @@ struct PlanUnit {  // one (request, KV head, row group) on the planner's cost ax
     int32_t max_cut;    // largest tile boundary at which a split may start so that the first row still sees a key
     int32_t last_cost;  // cost of the last (possibly short) tile
     int32_t overhead;   // fixed cost of the unit: query load, hand-off to the epilogue, output rows
+    int32_t pool_whole;   // 1: the unit is an item of the shared pool
 };
 
 struct PlanBuffers {  // caller-provided work arrays of plan_partition_core
@@ -39,12 +48,18 @@ struct PlanBuffers {  // caller-provided work arrays of plan_partition_core
 };
 
 int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads);
+// Items [cta_begin[c], cta_begin[c+1]) belong to CTA c; items [cta_begin[n_ctas], n_items) are the shared pool.
 int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads,
                         int32_t n_ctas, const PlanTuning &tune, const PlanBuffers &buf, int32_t *n_items_out,
                         int32_t *n_units_out, int32_t *n_partials_out);
+struct PlanScratch {  // work arrays of plan_partition that a caller may keep between calls
+    std::vector<PlanUnit> units;
+    std::vector<int64_t> start;
+};
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
-                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out);
+                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out,
+                   PlanScratch *scratch = nullptr);
 
 // ---- slot layout (private to the library) -----------------------------------------------------------
 // A slot's range is a sequence of tile blocks of XLLM_TILE_TOKENS tokens.  A tile block holds, for each
@@ -106,6 +121,9 @@ struct AttnLaunch {
     float *part_o;                // [n_partials][kMaxRows][D] fp32
     float *part_lse;              // [n_partials][kMaxRows]    (log2 domain)
     int32_t *counters;            // [n_partials] arrival counters of split units, zero between launches
+    uint32_t *pool_counter;       // claims made on the shared pools of all launches so far (never reset between launches)
+    uint32_t pool_base;           // ... its value when this launch starts: claim number t gets pool record t - pool_base
+    int32_t n_pool, pool_first;   // the pool: items[pool_first .. pool_first + n_pool)
     int32_t *error_flag;          // host-mapped; set non-zero when a bounded wait expires
     unsigned long long *trace;    // optional per-CTA cycle counters (debug), may be null
     int32_t n_q_heads, n_kv_heads, head_dim;

@@ -21,12 +21,14 @@ def binding():
 def check_plan(binding, kv, ql, hq, hkv, n_ctas):
     items, cta, n_units, n_parts = binding.plan_partition(kv, ql, hq, hkv, n_ctas)
     G = hq // hkv
-    assert cta[0] == 0 and cta[-1] == len(items) and np.all(np.diff(cta) >= 0)
+    assert cta[0] == 0 and cta[-1] <= len(items) and np.all(np.diff(cta) >= 0)
+    pool = items[cta[-1]:]          # claimed at run time by whichever CTA is done with its own run
+    assert len(pool) <= 8 * n_ctas
     cover = {}
     partial_ids = []
     loads = np.zeros(n_ctas, np.int64)
-    for c in range(n_ctas):
-        for it in items[cta[c]:cta[c + 1]]:
+    for c in range(n_ctas + 1):
+        for it in (items[cta[c]:cta[c + 1]] if c < n_ctas else pool):
             # cost axis of the planner: 8 per full tile, the unit's last tile in proportion to its 16-token steps,
             # plus 6 + 8 * rows / 16 per work item
             q_len_ = 1 if ql is None else int(ql[it.req])
@@ -37,7 +39,10 @@ def check_plan(binding, kv, ql, hq, hkv, n_ctas):
             if it.tile_end == nt:
                 tail_rows = min(T, -(-(vis - (nt - 1) * T) // 16) * 16)
                 cost += 4 + 8 * tail_rows // (2 * T) - 8
-            loads[c] += cost + 6 + 8 * it.n_q_tok * it.n_g // 16   # every piece pays the unit's fixed cost
+            if c < n_ctas:
+                loads[c] += cost + 6 + 8 * it.n_q_tok * it.n_g // 16   # every piece pays the unit's fixed cost
+            else:
+                assert it.partial_idx < 0 and it.tile_begin == 0 and it.tile_end == nt and 4 <= nt <= 64   # whole small units only
             key = (it.req, it.kv_head, it.q_tok0, it.g0)
             q_len = 1 if ql is None else int(ql[it.req])
             vis_last = int(kv[it.req]) - q_len + it.q_tok0 + it.n_q_tok

@@ -122,6 +122,24 @@ def test_named_decode_workload_fused(binding):
     gh.assert_parity(out, lse, *gh.oracle_batch(batch))
 
 
+def test_fused_append_with_items_from_the_shared_pool(binding):
+    """Small whole units are claimed at run time; in a fused launch the claiming CTA writes their new rows itself."""
+    import gpu_harness as gh
+
+    rng = np.random.default_rng(21)
+    lens, qls = [], []
+    for i in range(96):
+        qls.append(int(rng.integers(1, 5)))
+        lens.append(int(rng.integers(300, 900)) if i % 3 == 0 else int(rng.integers(2500, 4000)))
+    items, cta, _, _ = binding.plan_partition(lens, qls, 32, 8, 148)
+    pool = items[cta[-1]:]
+    assert len(pool) >= 32 and len(items) <= 8 * 148          # the case really has a pool and still fuses the append
+    batch = wl.custom_batch(415, 32, 8, 128, lens, qls)
+    out, lse, launches = run_fused(binding, batch)
+    assert launches == 0
+    gh.assert_parity(out, lse, *gh.oracle_batch(batch))
+
+
 def test_not_mapped_is_refused_before_anything_runs(binding):
     import gpu_harness as gh
 

@@ -16,6 +16,9 @@
  *     and state checks run before any kernel is launched.  An asynchronous CUDA error or a device
  *     side wait that gave up is reported by the next call (or xllm_sync_check) as XLLM_ERR_CUDA.
  *   - A context is bound to one device and is not thread safe; callers serialise.
+ *   - The attention calls of one context share its workspace (partial results, arrival and claim
+ *     counters): their kernels must not overlap on the GPU.  Calls on one stream never do; a caller
+ *     that moves a context from one stream to another orders the two streams itself (an event).
  *   - bf16 tensors are raw 16-bit patterns; all tensors are dense and row major.
  */
 #ifndef XLLM_ATTN_H

@@ -252,6 +252,72 @@ class Replica:
         t.cuda.current_stream().synchronize()                              # the caller reads the result every step
 
 
+def run_split(args):
+    """`--split P`: every sequence's KV is held as P parts in P ranges; a step is P partial-attention calls (what P ranks
+    would run side by side, here back to back on one GPU) and the log-sum-exp merge.  Shows what the split costs on top
+    of the unsplit step: a side measurement, not the headline."""
+    import torch
+
+    from paper_2510_14686_b200 import binding
+
+    torch.cuda.set_device(0)
+    name, P = args.workload, args.split
+    s = wl.SHAPES[name]
+    kv, ql = wl.draw_lengths(name)
+    B = len(kv)
+    copies = 2
+    page = 2 << 20
+    bounds = [[int(round((int(kv[r]) - int(ql[r])) * p / P)) for p in range(P)] + [int(kv[r])] for r in range(B)]
+    pages = sum(-(-(-(-(b[p + 1] - b[p]) // 64) * 64 * s.row_bytes) // page) + 1 for b in bounds for p in range(P)) * copies + 4
+    ctx = binding.Context(s.n_q_heads, s.n_kv_heads, s.head_dim, B * P * copies, int(kv.max()) + 64, pages * page, max_q_len=4)
+    gen = torch.Generator(device="cuda").manual_seed(s.seed)
+    slots = [[np.zeros(B, np.int32) for _ in range(P)] for _ in range(copies)]
+    for c in range(copies):
+        for r in range(B):
+            for p in range(P):
+                n_tok = bounds[r][p + 1] - bounds[r][p]
+                sl = ctx.kv_reserve(expected_tokens=n_tok)
+                ctx.kv_map_pages(sl, n_tok)
+                for t0 in range(0, n_tok, 1 << 15):
+                    n = min(n_tok - t0, 1 << 15)
+                    k = torch.randn((n, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+                    v = torch.randn((n, s.n_kv_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+                    ctx.kv_append([sl], [n], k, v)
+                slots[c][p][r] = sl
+    rows = int(ql.sum())
+    q = torch.randn((rows, s.n_q_heads, s.head_dim), generator=gen, device="cuda").to(torch.bfloat16)
+    outs = torch.empty((P, rows, s.n_q_heads, s.head_dim), dtype=torch.float32, device="cuda")
+    lses = torch.empty((P, rows, s.n_q_heads), dtype=torch.float32, device="cuda")
+    out = torch.zeros_like(q)
+    tails = [[int(p == P - 1)] * B for p in range(P)]
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step(i):
+        for p in range(P):
+            ctx.partial_attention(slots[i % copies][p], ql, tails[p], q, outs[p], lses[p], s.scale, stream)
+        ctx.merge_partials(outs, lses, out, None, stream)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    ctx.sync_check()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    ctx.sync_check()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    kv_bytes = int(kv.sum()) * s.row_bytes
+    print(json.dumps({"metric": METRIC, "value": int(kv.sum()) / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+                      "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"{name}, every sequence held as {P} parts: {P} partial-attention calls back to back + merge",
+                                 "kv_bytes_per_step_per_gpu": kv_bytes},
+                      "hbm_gbs_whole_step": kv_bytes / (ms * 1e-3) / 1e9, "gpu_launches": None}))
+
+
 def run_ours(args):
     import torch
 
@@ -398,11 +464,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=list(wl.SHAPES), default="decode")
+    ap.add_argument("--split", type=int, default=1, help="side measurement: every sequence held as this many parts (1 GPU)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     else:
-        run_ours(args)
+        run_split(args) if args.split > 1 else run_ours(args)
 
 
 if __name__ == "__main__":

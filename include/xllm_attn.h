@@ -278,6 +278,31 @@ xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_t *kv_range
                                          int32_t n_kv_heads, int32_t head_dim, const void *q, void *out, float *lse_out,
                                          float scale, void *cuda_stream);
 
+/* ---- sequences split over several ranges (or GPUs) --------------------------------------------------------------
+ * The report's inter-DP-group migration moves part of a long sequence's KV blocks to another group, lets it compute
+ * attention over them, and gathers the external results with an aggregation operator (section "Hierarchical DP Load
+ * Balance", partial migration at block granularity).  The two calls below are that pair: each holder of a part runs
+ * xllm_partial_attention over its part, the caller brings the partial results together (on one GPU: nothing to do;
+ * across GPUs: an all-gather of a few KB per request), and xllm_merge_partials merges them by log-sum-exp. */
+
+/* Attention over the part of each sequence that slots[i] holds.  Like xllm_verify_attention, except:
+ *   - causal_tail: host int32 [n_req] or NULL (= all 1).  1: the range ends with the request's q_lens[i] newest
+ *     tokens (the query tokens themselves, causal among them) -- the part that holds the end of the sequence.
+ *     0: an older part; every one of its kv_len >= 1 tokens is visible to every query token.
+ *   - out_part: device fp32 [sum q_lens, H_q, D], softmax-normalised within the part (zeros where the part holds no
+ *     visible key); lse_part: device fp32 [sum q_lens, H_q], natural log of the part's softmax denominator
+ *     (-inf where the part holds no visible key).  Both are required. */
+xllm_status xllm_partial_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
+                                   const int32_t *causal_tail, const void *q, float *out_part, float *lse_part, float scale,
+                                   void *cuda_stream);
+
+/* Merge n_parts partial results of the same n_rows query tokens: out_parts device fp32 [n_parts, n_rows, H_q, D],
+ * lse_parts device fp32 [n_parts, n_rows, H_q] (the layout an all-gather of the calls' outputs produces).
+ * out: device bf16 [n_rows, H_q, D]; lse_out: device fp32 [n_rows, H_q] or NULL.  Parts are added in index order
+ * (repeatable bit for bit); a part with lse = -inf has weight 0 whatever its values. */
+xllm_status xllm_merge_partials(xllm_ctx *ctx, int32_t n_parts, int64_t n_rows, const float *out_parts, const float *lse_parts,
+                                void *out, float *lse_out, void *cuda_stream);
+
 /* ---- work partition (host only; exposed so that it can be checked without a GPU) ---------------------------- */
 
 /* Split the step's KV tile blocks into per-CTA runs of near-equal cost (hierarchical DP load balance,

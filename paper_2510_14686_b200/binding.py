@@ -101,6 +101,8 @@ EXPORTS = {
     "xllm_append_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_decode_attention_static": (ctypes.c_int32, [ctypes.c_int32, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                        _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_partial_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_merge_partials": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, _vp, _vp, _vp, _vp, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.POINTER(WorkItem), ctypes.c_int32, _i32p, _i32p, _i32p, _i32p]),
     "xllm_get_stats": (ctypes.c_int32, [_ctxp, ctypes.POINTER(Stats)]),
@@ -296,6 +298,19 @@ class Context:
         s, ql = _i32(slots), _i32(q_lens)
         self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(q), _ptr(out),
                                                _ptr(lse_out), scale, _stream(stream)))
+
+    def partial_attention(self, slots, q_lens, causal_tail, q, out_part, lse_part, scale: float = 1.0, stream=None):
+        """Attention over the part of each sequence that its slot holds: fp32 ``out_part`` and ``lse_part`` for a later merge."""
+        s, ql = _i32(slots), _i32(q_lens)
+        ct = _i32(causal_tail) if causal_tail is not None else None
+        self._check(_lib.xllm_partial_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data,
+                                                ct.ctypes.data if ct is not None else None, _ptr(q), _ptr(out_part),
+                                                _ptr(lse_part), scale, _stream(stream)))
+
+    def merge_partials(self, out_parts, lse_parts, out, lse_out=None, stream=None):
+        """``out_parts`` fp32 [n_parts, rows, H_q, D], ``lse_parts`` fp32 [n_parts, rows, H_q] -> bf16 ``out`` (+ ``lse_out``)."""
+        self._check(_lib.xllm_merge_partials(self._ctx, int(out_parts.shape[0]), int(out_parts.shape[1]), _ptr(out_parts),
+                                             _ptr(lse_parts), _ptr(out), _ptr(lse_out), _stream(stream)))
 
     def append_decode_attention(self, slots, k_new, v_new, q, out, lse_out=None, scale: float = 1.0, stream=None):
         s = _i32(slots)

@@ -266,7 +266,8 @@ void stop_worker(xllm_ctx *ctx) {
 // request's rows fit one row group, else by a separate append launch) and then attends over the grown ranges.
 xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
                            void *out, float *lse_out, float scale, void *cuda_stream, const char *who,
-                           const void *k_new = nullptr, const void *v_new = nullptr) {
+                           const void *k_new = nullptr, const void *v_new = nullptr, const int32_t *causal_tail = nullptr,
+                           bool out_f32 = false) {
     if (!ctx) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     const bool with_append = k_new != nullptr || v_new != nullptr;
@@ -302,15 +303,16 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
             q_rows += ql;
             continue;
         }
-        if (s.kv_len < ql)
+        if (s.kv_len < ((!causal_tail || causal_tail[i]) ? ql : 1))
             return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(slots[i]) + " holds " +
-                                                   std::to_string(s.kv_len) + " tokens, fewer than q_len " + std::to_string(ql));
+                                                   std::to_string(s.kv_len) + " tokens, fewer than the call needs (q_len " +
+                                                   std::to_string(ql) + ")");
         ctx->kv_lens[(size_t)i] = s.kv_len;
         q_rows += ql;
     }
     int32_t n_units = 0, n_partials = 0;
     if (plan_partition(n_req, ctx->kv_lens.data(), q_lens, ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, ctx->sm_count, ctx->tune,
-                       ctx->items, ctx->cta_begin, &n_units, &n_partials, &ctx->plan_scratch) != 0)
+                       ctx->items, ctx->cta_begin, &n_units, &n_partials, &ctx->plan_scratch, causal_tail) != 0)
         return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
     const int32_t n_items = (int32_t)ctx->items.size();
     if (n_items > ctx->max_items || n_partials > ctx->max_partials)
@@ -372,12 +374,14 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         di[i].tile_begin = w.tile_begin;
         di[i].tile_end = w.tile_end;
         const int64_t kv_now = ctx->kv_lens[(size_t)w.req];  // tokens in the range when the kernel reads it
-        di[i].kv_end = (int32_t)kv_now - ql + w.q_tok0 + w.n_q_tok;
+        const bool tail = !causal_tail || causal_tail[w.req];
+        di[i].kv_end = tail ? (int32_t)kv_now - ql + w.q_tok0 + w.n_q_tok : (int32_t)kv_now;
+        di[i].flags = tail ? 0 : kItemAllVisible;
         di[i].head0 = (int16_t)(w.kv_head * G + w.g0);
         di[i].n_q_tok = (uint8_t)w.n_q_tok;
         di[i].n_g = (uint8_t)w.n_g;
         di[i].part_first = w.part_first;
-        di[i].n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
+        di[i].n_parts = (int16_t)(w.n_parts <= kFuseMaxParts ? w.n_parts : 0);
         di[i].new_row = q_row0[(size_t)w.req];
         di[i].n_new = (fuse && w.tile_end == (kv_now + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS) ? ql : 0;
     }
@@ -405,6 +409,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.n_q_heads = ctx->cfg.n_q_heads;
     al.n_kv_heads = ctx->cfg.n_kv_heads;
     al.head_dim = ctx->cfg.head_dim;
+    al.out_f32 = out_f32 ? 1 : 0;
     al.scale_log2 = scale * 1.4426950408889634f;
     al.n_ctas = ctx->sm_count;
     al.debug_stall_cta = -1;
@@ -432,6 +437,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         cl.lse_out = lse_out;
         cl.n_q_heads = ctx->cfg.n_q_heads;
         cl.head_dim = ctx->cfg.head_dim;
+        cl.out_f32 = out_f32 ? 1 : 0;
         time_begin(ctx, 1, stream);
         e = launch_combine(cl, stream);
         time_end(ctx, stream);
@@ -880,6 +886,33 @@ xllm_status xllm_append_verify_attention(xllm_ctx *ctx, int32_t n_req, const int
     if (ctx && (!q_lens || !k_new || !v_new))
         return fail(ctx, XLLM_ERR_INVALID, "append_verify_attention: q_lens, k_new and v_new must be non-null");
     return attention_impl(ctx, n_req, slots, q_lens, q, out, lse_out, scale, cuda_stream, "append_verify_attention", k_new, v_new);
+}
+
+xllm_status xllm_partial_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,
+                                   const int32_t *causal_tail, const void *q, float *out_part, float *lse_part, float scale,
+                                   void *cuda_stream) {
+    if (ctx && (!q_lens || !lse_part)) return fail(ctx, XLLM_ERR_INVALID, "partial_attention: q_lens and lse_part must be non-null");
+    return attention_impl(ctx, n_req, slots, q_lens, q, out_part, lse_part, scale, cuda_stream, "partial_attention", nullptr, nullptr,
+                          causal_tail, true);
+}
+
+xllm_status xllm_merge_partials(xllm_ctx *ctx, int32_t n_parts, int64_t n_rows, const float *out_parts, const float *lse_parts,
+                                void *out, float *lse_out, void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "merge_partials: context is host-only, no GPU work possible");
+    const xllm_status st = check_device_flag(ctx);
+    if (st != XLLM_OK) return st;
+    if (n_parts < 1 || n_rows < 1 || !out_parts || !lse_parts || !out)
+        return fail(ctx, XLLM_ERR_INVALID, "merge_partials: n_parts, n_rows >= 1 and non-null device pointers");
+    if ((reinterpret_cast<uintptr_t>(out_parts) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, "merge_partials: out_parts and out must be 16-byte aligned");
+    if (n_rows * ctx->cfg.n_q_heads > INT32_MAX) return fail(ctx, XLLM_ERR_UNSUPPORTED, "merge_partials: too many rows for one launch");
+    const int e = launch_merge_parts(n_parts, n_rows, ctx->cfg.n_q_heads, ctx->cfg.head_dim, out_parts, lse_parts, out, lse_out,
+                                     cuda_stream);
+    if (e) return cuda_fail(ctx, "launching the merge kernel", e);
+    ++ctx->st.kernel_launches;
+    return XLLM_OK;
 }
 
 xllm_status xllm_plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,

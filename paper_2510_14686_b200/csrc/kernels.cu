@@ -165,6 +165,16 @@ __device__ __forceinline__ void group_bar(int group) {
     asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
 }
 
+// Four adjacent output columns of one (query token, head) row: bf16 for a final result, fp32 for a partial one that
+// the caller merges later (xllm_partial_attention).
+template <int D>
+__device__ __forceinline__ void store_out4(void *out, int out_f32, int64_t off, int c4, float x, float y, float z, float w) {
+    if (out_f32)
+        *reinterpret_cast<float4 *>(static_cast<float *>(out) + off * D + c4 * 4) = make_float4(x, y, z, w);
+    else
+        *reinterpret_cast<uint2 *>(static_cast<char *>(out) + off * (D * 2) + c4 * 8) = make_uint2(pack_bf16(x, y), pack_bf16(z, w));
+}
+
 // ---- split-KV attention ---------------------------------------------------------------------------------
 // Warp roles: 0-7 consumers (two groups of four taking alternate tiles), 8 producer (bulk copies), 9-11 epilogue
 // (merge the two group states of a finished item and write its result while the consumers go on).
@@ -604,7 +614,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     break;
                 ++n_done;
                 const int n_rows = it.n_q_tok * it.n_g;
-                const int row_limit0 = it.kv_end - it.n_q_tok + 1;
+                const bool all_visible = (it.flags & kItemAllVisible) != 0;  // an older part of a longer sequence: no causal tail
+                const int row_limit0 = all_visible ? it.kv_end : it.kv_end - it.n_q_tok + 1;
                 const uint32_t seq = item_seq + i, qb = seq & 1, qph = (seq >> 1) & 1;
                 uint32_t qf[D / 16][4];
                 unsigned long long t0 = TRACE ? clock64() : 0ull;
@@ -623,8 +634,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_qempty + qb * 8);
 
-                const int limit_lo = (g8 < n_rows) ? row_limit0 + g8 / it.n_g : 0;
-                const int limit_hi = (g8 + 8 < n_rows) ? row_limit0 + (g8 + 8) / it.n_g : 0;
+                const int limit_lo = (g8 < n_rows) ? row_limit0 + (all_visible ? 0 : g8 / it.n_g) : 0;
+                const int limit_hi = (g8 + 8 < n_rows) ? row_limit0 + (all_visible ? 0 : (g8 + 8) / it.n_g) : 0;
                 const bool half = n_rows <= 8;
                 float o[D / 32][4];
 #pragma unroll
@@ -768,8 +779,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     } else {
                         const int ti = row / it.n_g, gi = row - ti * it.n_g;
                         const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
-                        *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
-                            make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+                        store_out4<D>(p.out, p.out_f32, off, c4, acc.x, acc.y, acc.z, acc.w);
                         if (c4 == 0 && p.lse_out) p.lse_out[off] = lse_row * 0.69314718055994531f;
                     }
                 }
@@ -834,8 +844,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                                 const float inv = (W > 0.f) ? 1.f / W : 0.f;
                                 const int ti = row / it.n_g, gi = row - ti * it.n_g;
                                 const int64_t off = ((int64_t)it.q_row + ti) * p.n_q_heads + it.head0 + gi;
-                                *reinterpret_cast<uint2 *>(static_cast<char *>(p.out) + off * (D * 2) + c4 * 8) =
-                                    make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                                store_out4<D>(p.out, p.out_f32, off, c4, acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
                                 if (c4 == 0 && p.lse_out)
                                     p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
                             }
@@ -931,8 +940,44 @@ __global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
     }
     const int ti = row / d.n_g, gi = row - ti * d.n_g;
     const int64_t off = (int64_t)(d.out_row0 + ti) * p.n_q_heads + d.head0 + gi;
-    static_cast<__nv_bfloat16 *>(p.out)[off * D + col] = __float2bfloat16_rn(W > 0.f ? acc / W : 0.f);
+    const float res = W > 0.f ? acc / W : 0.f;
+    if (p.out_f32)
+        static_cast<float *>(p.out)[off * D + col] = res;
+    else
+        static_cast<__nv_bfloat16 *>(p.out)[off * D + col] = __float2bfloat16_rn(res);
     if (col == 0 && p.lse_out) p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
+}
+
+// ---- merge of partial results computed over parts of longer sequences (possibly on other GPUs) --------------
+// out_parts fp32 [n_parts][rows][H_q][D], each normalised within its part; lse_parts fp32 [n_parts][rows][H_q], natural
+// log, -inf where the part held no visible key.  One block per (row, head); parts are added in part order.
+template <int D>
+__global__ void __launch_bounds__(D / 4) merge_parts_kernel(int n_parts, int64_t n_rows_heads, const float *__restrict__ out_parts,
+                                                           const float *__restrict__ lse_parts, __nv_bfloat16 *__restrict__ out,
+                                                           float *__restrict__ lse_out) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int64_t rh = blockIdx.x;
+    const int c4 = threadIdx.x;
+    float M = -INFINITY;
+    for (int s = 0; s < n_parts; ++s) M = fmaxf(M, lse_parts[s * n_rows_heads + rh]);
+    const float Ms = (M == -INFINITY) ? 0.f : M;
+    float W = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < n_parts; ++s) {
+        const float w = expf(lse_parts[s * n_rows_heads + rh] - Ms);
+        const float4 v = reinterpret_cast<const float4 *>(out_parts + (s * n_rows_heads + rh) * D)[c4];
+        W += w;
+        if (w > 0.f) {  // (a part without visible keys may hold anything)
+            acc.x += w * v.x;
+            acc.y += w * v.y;
+            acc.z += w * v.z;
+            acc.w += w * v.w;
+        }
+    }
+    const float inv = W > 0.f ? 1.f / W : 0.f;
+    *reinterpret_cast<uint2 *>(out + rh * D + c4 * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+    if (c4 == 0 && lse_out) lse_out[rh] = W > 0.f ? M + logf(W) : -INFINITY;
 }
 
 // ---- append ("write_kvcache") and its inverse --------------------------------------------------------------
@@ -1035,6 +1080,18 @@ int launch_combine(const CombineLaunch &p, void *stream) {
     dim3 grid(p.n_units, kMaxRows);
     if (p.head_dim == 128) return (int)launch_pdl(combine_kernel<128>, grid, dim3(128), 0, st, p);
     return (int)launch_pdl(combine_kernel<64>, grid, dim3(64), 0, st, p);
+}
+
+int launch_merge_parts(int32_t n_parts, int64_t rows, int32_t n_q_heads, int32_t head_dim, const float *out_parts,
+                       const float *lse_parts, void *out, float *lse_out, void *stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t rh = rows * n_q_heads;
+    dim3 grid((unsigned)rh);
+    if (head_dim == 128)
+        return (int)launch_pdl(merge_parts_kernel<128>, grid, dim3(32), 0, st, (int)n_parts, rh, out_parts, lse_parts,
+                               static_cast<__nv_bfloat16 *>(out), lse_out);
+    return (int)launch_pdl(merge_parts_kernel<64>, grid, dim3(16), 0, st, (int)n_parts, rh, out_parts, lse_parts,
+                           static_cast<__nv_bfloat16 *>(out), lse_out);
 }
 
 int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *k_new, const void *v_new,

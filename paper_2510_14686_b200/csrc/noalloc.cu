@@ -162,7 +162,8 @@ extern "C" xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_
         d.n_q_tok = (uint8_t)w.n_q_tok;
         d.n_g = (uint8_t)w.n_g;
         d.part_first = w.part_first;
-        d.n_parts = w.n_parts <= kFuseMaxParts ? w.n_parts : 0;
+        d.n_parts = (int16_t)(w.n_parts <= kFuseMaxParts ? w.n_parts : 0);
+        d.flags = 0;
         d.new_row = d.n_new = 0;
     }
 

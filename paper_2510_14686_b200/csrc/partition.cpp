@@ -33,7 +33,8 @@ int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads
 
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
-                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out, PlanScratch *scratch) {
+                   std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out, PlanScratch *scratch,
+                   const int32_t *causal_tail) {
     const int64_t n_units = plan_count_units(n_req, q_lens, n_q_heads, n_kv_heads);
     if (n_units < 0 || n_ctas < 1 || n_units > INT32_MAX / 2) return -1;
     PlanScratch local;
@@ -45,7 +46,7 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
     PlanBuffers buf{sc.units.data(), sc.start.data(), (int32_t)n_units, items.data(), (int32_t)items.size(), cta_begin.data()};
     int32_t n_items = 0;
     const int rc = plan_partition_core(n_req, kv_lens, q_lens, n_q_heads, n_kv_heads, n_ctas, tune, buf, &n_items, n_units_out,
-                                       n_partials_out);
+                                       n_partials_out, causal_tail);
     items.resize(rc == 0 ? (size_t)n_items : 0);
     return rc;
 }
@@ -54,7 +55,7 @@ int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens,
 // array is too small.
 int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads,
                         int32_t n_ctas, const PlanTuning &tune, const PlanBuffers &buf, int32_t *n_items_out,
-                        int32_t *n_units_out, int32_t *n_partials_out) {
+                        int32_t *n_units_out, int32_t *n_partials_out, const int32_t *causal_tail) {
     if (n_req < 1 || n_ctas < 1 || n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads) return -1;
     const int32_t G = n_q_heads / n_kv_heads;
     const int32_t T = XLLM_TILE_TOKENS;
@@ -73,21 +74,22 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     for (int32_t r = 0; r < n_req; ++r) {
         const int64_t kv = kv_lens[r];
         const int32_t ql = q_lens ? q_lens[r] : 1;
-        if (ql < 1 || kv < ql || kv > INT32_MAX) return -1;
+        if (ql < 1 || kv < 1 || ((!causal_tail || causal_tail[r]) && kv < ql) || kv > INT32_MAX) return -1;
         for (int32_t h = 0; h < n_kv_heads; ++h) {
             if (G <= kMaxRows) {
                 const int32_t per = std::max(1, kMaxRows / G);  // query tokens per row group
                 for (int32_t t0 = 0; t0 < ql; t0 += per) {
                     const int32_t nt = std::min(per, ql - t0);
-                    const int64_t vis_last = kv - ql + t0 + nt;  // keys visible to the last row
-                    const int64_t vis_first = kv - ql + t0 + 1;  // keys visible to the first row
+                    const bool tail = !causal_tail || causal_tail[r];
+                    const int64_t vis_last = tail ? kv - ql + t0 + nt : kv;  // keys visible to the last row
+                    const int64_t vis_first = tail ? kv - ql + t0 + 1 : kv;  // keys visible to the first row
                     Unit u{r, h, (int16_t)t0, (int16_t)nt, 0, (int16_t)G, (int32_t)((vis_last + T - 1) / T),
                            (int32_t)((vis_first - 1) / T), 0, 0, 0};
                     units.push_back(u);
                 }
             } else {
                 for (int32_t t0 = 0; t0 < ql; ++t0) {
-                    const int64_t vis = kv - ql + t0 + 1;
+                    const int64_t vis = (!causal_tail || causal_tail[r]) ? kv - ql + t0 + 1 : kv;
                     for (int32_t g0 = 0; g0 < G; g0 += kMaxRows) {
                         Unit u{r, h, (int16_t)t0, 1, (int16_t)g0, (int16_t)std::min(kMaxRows, G - g0),
                                (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T), 0, 0, 0};
@@ -151,7 +153,8 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     start[0] = 0;
     for (int32_t u = 0; u < U; ++u) {
         Unit &un = units[u];
-        const int64_t vis_last = kv_lens[un.req] - (q_lens ? q_lens[un.req] : 1) + un.q_tok0 + un.n_q_tok;
+        const int64_t vis_last = (!causal_tail || causal_tail[un.req]) ? kv_lens[un.req] - (q_lens ? q_lens[un.req] : 1) + un.q_tok0 + un.n_q_tok
+                                                                      : kv_lens[un.req];
         const int32_t tail_rows = (int32_t)std::min<int64_t>(T, ((vis_last - (int64_t)(un.n_tiles - 1) * T) + 15) / 16 * 16);
         un.last_cost = tune.tile_cost / 2 + tune.tile_cost * tail_rows / (2 * T);  // half fixed, half by volume
         un.overhead = tune.unit_overhead + tune.row_overhead * un.n_q_tok * un.n_g / kMaxRows;

@@ -49,9 +49,11 @@ struct PlanBuffers {  // caller-provided work arrays of plan_partition_core
 
 int64_t plan_count_units(int32_t n_req, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads);
 // Items [cta_begin[c], cta_begin[c+1]) belong to CTA c; items [cta_begin[n_ctas], n_items) are the shared pool.
+// causal_tail (may be null = all 1): 0 for a request whose range holds an older part of a longer sequence, so that
+// every key is visible to every query token; 1 when the newest q_len tokens of the range are the query tokens.
 int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads, int32_t n_kv_heads,
                         int32_t n_ctas, const PlanTuning &tune, const PlanBuffers &buf, int32_t *n_items_out,
-                        int32_t *n_units_out, int32_t *n_partials_out);
+                        int32_t *n_units_out, int32_t *n_partials_out, const int32_t *causal_tail = nullptr);
 struct PlanScratch {  // work arrays of plan_partition that a caller may keep between calls
     std::vector<PlanUnit> units;
     std::vector<int64_t> start;
@@ -59,7 +61,7 @@ struct PlanScratch {  // work arrays of plan_partition that a caller may keep be
 int plan_partition(int32_t n_req, const int64_t *kv_lens, const int32_t *q_lens, int32_t n_q_heads,
                    int32_t n_kv_heads, int32_t n_ctas, const PlanTuning &tune, std::vector<xllm_work_item> &items,
                    std::vector<int32_t> &cta_begin, int32_t *n_units_out, int32_t *n_partials_out,
-                   PlanScratch *scratch = nullptr);
+                   PlanScratch *scratch = nullptr, const int32_t *causal_tail = nullptr);
 
 // ---- slot layout (private to the library) -----------------------------------------------------------
 // A slot's range is a sequence of tile blocks of XLLM_TILE_TOKENS tokens.  A tile block holds, for each
@@ -77,6 +79,8 @@ constexpr int32_t kMaxCtas = 160;  // upper bound on the persistent grid (B200: 
 
 constexpr int32_t kFuseMaxParts = 4;  // units split into at most this many pieces are merged inside the attention kernel
 
+constexpr int16_t kItemAllVisible = 1;
+
 struct DevItem {            // one work item, resolved on the host against the slot table (48 bytes)
     uint64_t kv;            // address of the item's KV head inside tile block 0 of the slot's range
     int32_t q_row;          // first row of the item's query group in q / out  (request row + q_tok0)
@@ -86,7 +90,8 @@ struct DevItem {            // one work item, resolved on the host against the s
     int16_t head0;          // first query head of the group (kv_head * G + g0)
     uint8_t n_q_tok, n_g;   // rows = n_q_tok * n_g <= kMaxRows
     int32_t part_first;     // partial slot of the unit's first piece (also the index of the unit's arrival counter)
-    int32_t n_parts;        // pieces of the unit if the last piece to finish merges them in-kernel; 0 = combine kernel
+    int16_t n_parts;        // pieces of the unit if the last piece to finish merges them in-kernel; 0 = combine kernel
+    int16_t flags;          // kItemAllVisible: every key of the range is visible to every query row (no causal tail)
     int32_t new_row;        // fused append: first row of the request's new tokens in k_new / v_new ...
     int32_t n_new;          // ... and how many this item must write into the range before reading its last tiles (else 0)
 };
@@ -127,6 +132,7 @@ struct AttnLaunch {
     int32_t *error_flag;          // host-mapped; set non-zero when a bounded wait expires
     unsigned long long *trace;    // optional per-CTA cycle counters (debug), may be null
     int32_t n_q_heads, n_kv_heads, head_dim;
+    int32_t out_f32;              // 1: `out` is fp32 (a partial result for a later merge) instead of bf16
     float scale_log2;             // scale * log2(e)
     int32_t n_ctas;
     int32_t debug_stall_cta;      // -1; else that CTA arms the V half of its first tile but never copies it (timeout test)
@@ -142,6 +148,7 @@ struct CombineLaunch {
     void *out;
     float *lse_out;
     int32_t n_q_heads, head_dim;
+    int32_t out_f32;
 };
 
 constexpr int32_t kTraceWords = 16;  // per-CTA words of the optional trace buffer
@@ -151,6 +158,8 @@ int attention_smem_bytes(int32_t head_dim);
 int configure_kernels(int32_t head_dim);  // cudaFuncSetAttribute for the dynamic shared memory; returns cudaError
 int launch_attention(const AttnLaunch &p, void *stream);
 int launch_combine(const CombineLaunch &p, void *stream);
+int launch_merge_parts(int32_t n_parts, int64_t rows, int32_t n_q_heads, int32_t head_dim, const float *out_parts,
+                       const float *lse_parts, void *out, float *lse_out, void *stream);
 int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *k_new, const void *v_new,
                   int32_t n_kv_heads, int32_t head_dim, void *stream);
 int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,

@@ -504,9 +504,10 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         drv = make_cuda_driver(&derr);
         if (!drv) return bad(XLLM_ERR_CUDA, derr);
     }
-    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece[,pieces_first[,pool_pct[,pool_min[,fuse_max]]]]": planner override (tuning aid)
-        int a, b, c, d, f = ctx->tune.pieces_first, g = ctx->tune.pool_pct, h = ctx->tune.pool_min_tiles, k = ctx->tune.fuse_max_items_per_cta;
-        if (std::sscanf(t, "%d,%d,%d,%d,%d,%d,%d,%d", &a, &b, &c, &d, &f, &g, &h, &k) >= 4 && a > 0 && b >= 0 && c >= 0 && d >= 1 && g >= 0 &&
+    if (const char *t = std::getenv("XLLM_PLAN_TUNE")) {  // "tile,unit,row,min_piece[,pieces_first[,pool_pct[,pool_min[,fuse_max[,pool_share_div]]]]]": planner override (tuning aid)
+        int a, b, c, d, f = ctx->tune.pieces_first, g = ctx->tune.pool_pct, h = ctx->tune.pool_min_tiles, k = ctx->tune.fuse_max_items_per_cta,
+            m = ctx->tune.pool_share_div;
+        if (std::sscanf(t, "%d,%d,%d,%d,%d,%d,%d,%d,%d", &a, &b, &c, &d, &f, &g, &h, &k, &m) >= 4 && a > 0 && b >= 0 && c >= 0 && d >= 1 && g >= 0 &&
             g <= 50 && h >= 1) {
             ctx->tune.tile_cost = a;
             ctx->tune.unit_overhead = b;
@@ -516,6 +517,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
             ctx->tune.pool_pct = g;
             ctx->tune.pool_min_tiles = h;
             ctx->tune.fuse_max_items_per_cta = k;
+            ctx->tune.pool_share_div = m > 0 ? m : 8;
         }
     }
     ctx->xt.reset(new XTensor(std::move(drv), cfg->device, cfg->max_slots, cfg->max_seq_len, row_bytes));

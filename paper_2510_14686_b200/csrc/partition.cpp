@@ -126,7 +126,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
         const int64_t max_items = (int64_t)kPoolMaxPerCta * n_ctas;
         constexpr int32_t kMaxWhole = 64;
         const int32_t lo = std::max(1, tune.pool_min_tiles);
-        const int32_t hi = (int32_t)std::min<int64_t>(kMaxWhole, share / 8);  // (much shorter than a CTA's run, or it evens out nothing)
+        const int32_t hi = (int32_t)std::min<int64_t>(kMaxWhole, share / std::max(1, tune.pool_share_div));  // (much shorter than a CTA's run)
         int32_t quota[kMaxWhole + 1] = {0};  // units of each size: first how many there are, then how many go to the pool
         for (int32_t u = 0; u < U && target_tiles > 0; ++u)
             if (units[u].n_tiles >= lo && units[u].n_tiles <= hi) ++quota[units[u].n_tiles];

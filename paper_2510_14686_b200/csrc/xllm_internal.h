@@ -24,6 +24,7 @@ struct PlanTuning {
     // verification batch; batches of many short requests gain up to 15.
     int32_t pool_pct = 8;
     int32_t pool_min_tiles = 4;   // units smaller than this stay with a CTA: claiming costs about as much as they do
+    int32_t pool_share_div = 8;   // ... and units larger than a CTA's share / this are too coarse to even anything out
 };
 
 constexpr int32_t kPoolMaxPerCta = 8;  // the shared pool holds at most this many pieces per CTA

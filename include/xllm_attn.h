@@ -278,6 +278,32 @@ xllm_status xllm_decode_attention_static(int32_t n_req, const uint64_t *kv_range
                                          int32_t n_kv_heads, int32_t head_dim, const void *q, void *out, float *lse_out,
                                          float scale, void *cuda_stream);
 
+/* ---- graph mode: a step that can be captured once and replayed with other lengths ----------------------------------
+ * The report's adaptive graph mode captures kernels once and replays them with parameterised dimensions.  For this
+ * path: the step's launch records (work list, per-CTA ranges, lengths) live in host memory mapped into the device; the
+ * kernels read them when they start, so their launch parameters never change and a CUDA graph that contains them (a
+ * whole decoder layer, say) stays valid while batch composition and context lengths change.
+ *
+ *   xllm_graph_step_create   binds the step's device buffers once: q [rows, H_q, D] bf16, out likewise, lse_out fp32
+ *                            [rows, H_q] or NULL, k_new / v_new [rows, H_kv, D] bf16 or both NULL (no append); the
+ *                            caller keeps them alive and large enough for every batch it plans.  Allocates the record.
+ *   xllm_graph_step_plan     host only, NOT captured: partitions the work for the slots' current lengths (+ q_len new
+ *                            rows per request when k_new is bound, as xllm_append_verify_attention does; q_lens NULL =
+ *                            all 1) and rewrites the record; updates the slots' kv_len.  Call it before each replay,
+ *                            and only when no replay that uses this handle can still be running (it rewrites memory
+ *                            the kernels read).  UNSUPPORTED if the batch would need a separate append launch.
+ *   xllm_graph_step_launch   launches the step on cuda_stream: capturable; always the same two kernels with the same
+ *                            parameters (the second, the merge of heavily split sequences, exits at once when the
+ *                            plan has none).  One launch or replay per plan when k_new is bound (a second would append
+ *                            the same rows again, harmlessly, and attend to the same lengths).
+ *   xllm_graph_step_destroy  waits for the device and frees the record.
+ * Graph-mode launches share the context's workspace with the other attention calls (see the conventions above). */
+xllm_status xllm_graph_step_create(xllm_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, float *lse_out,
+                                   float scale, int32_t *handle_out);
+xllm_status xllm_graph_step_plan(xllm_ctx *ctx, int32_t handle, int32_t n_req, const int32_t *slots, const int32_t *q_lens);
+xllm_status xllm_graph_step_launch(xllm_ctx *ctx, int32_t handle, void *cuda_stream);
+xllm_status xllm_graph_step_destroy(xllm_ctx *ctx, int32_t handle);
+
 /* ---- sequences split over several ranges (or GPUs) --------------------------------------------------------------
  * The report's inter-DP-group migration moves part of a long sequence's KV blocks to another group, lets it compute
  * attention over them, and gathers the external results with an aggregation operator (section "Hierarchical DP Load

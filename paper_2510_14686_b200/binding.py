@@ -101,6 +101,10 @@ EXPORTS = {
     "xllm_append_verify_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_decode_attention_static": (ctypes.c_int32, [ctypes.c_int32, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                        _vp, _vp, _vp, ctypes.c_float, _vp]),
+    "xllm_graph_step_create": (ctypes.c_int32, [_ctxp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _i32p]),
+    "xllm_graph_step_plan": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int32, _vp, _vp]),
+    "xllm_graph_step_launch": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp]),
+    "xllm_graph_step_destroy": (ctypes.c_int32, [_ctxp, ctypes.c_int32]),
     "xllm_partial_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_merge_partials": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, _vp, _vp, _vp, _vp, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
@@ -298,6 +302,24 @@ class Context:
         s, ql = _i32(slots), _i32(q_lens)
         self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(q), _ptr(out),
                                                _ptr(lse_out), scale, _stream(stream)))
+
+    # -- graph mode --
+    def graph_step_create(self, q, out, lse_out=None, k_new=None, v_new=None, scale: float = 1.0) -> int:
+        h = ctypes.c_int32(-1)
+        self._check(_lib.xllm_graph_step_create(self._ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse_out), scale,
+                                                ctypes.byref(h)))
+        return h.value
+
+    def graph_step_plan(self, handle: int, slots, q_lens=None):
+        s = _i32(slots)
+        ql = _i32(q_lens) if q_lens is not None else None
+        self._check(_lib.xllm_graph_step_plan(self._ctx, handle, len(s), s.ctypes.data, ql.ctypes.data if ql is not None else None))
+
+    def graph_step_launch(self, handle: int, stream=None):
+        self._check(_lib.xllm_graph_step_launch(self._ctx, handle, _stream(stream)))
+
+    def graph_step_destroy(self, handle: int):
+        self._check(_lib.xllm_graph_step_destroy(self._ctx, handle))
 
     def partial_attention(self, slots, q_lens, causal_tail, q, out_part, lse_part, scale: float = 1.0, stream=None):
         """Attention over the part of each sequence that its slot holds: fp32 ``out_part`` and ``lse_part`` for a later merge."""

@@ -45,6 +45,20 @@ struct PremapJob {
     int64_t min_tokens;
 };
 
+// Graph mode: one step whose launch parameters never change.  The launch records and the work list sit in one buffer of
+// pinned host memory mapped into the device; xllm_graph_step_plan rewrites it, xllm_graph_step_launch launches kernels that
+// read it.
+struct GraphStep {
+    char *h_buf = nullptr, *d_buf = nullptr;
+    CombineLaunch *d_cl = nullptr;  // device copy of the second kernel's record, written by the first
+    size_t bytes = 0;
+    const void *q = nullptr, *k_new = nullptr, *v_new = nullptr;
+    void *out = nullptr;
+    float *lse_out = nullptr;
+    float scale = 1.f;
+    bool planned = false;
+};
+
 struct xllm_ctx {
     // One lock serialises every entry point and the pre-mapping worker (recursive: the fused append falls back to
     // xllm_kv_append from inside an attention call).
@@ -87,6 +101,7 @@ struct xllm_ctx {
     uint64_t scratch_va = 0;
 
     PlanScratch plan_scratch;
+    std::vector<GraphStep *> graph_steps;  // by handle; null after destroy
     uint32_t pool_base = 0;       // claims made on the shared pools of all launches so far (mirrors the device counter)
     int32_t inject_timeouts = 0;  // attention launches still to be made with one stalled copy (test hook)
     bool profiling = false;
@@ -267,7 +282,7 @@ void stop_worker(xllm_ctx *ctx) {
 xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q,
                            void *out, float *lse_out, float scale, void *cuda_stream, const char *who,
                            const void *k_new = nullptr, const void *v_new = nullptr, const int32_t *causal_tail = nullptr,
-                           bool out_f32 = false) {
+                           bool out_f32 = false, GraphStep *gs = nullptr) {
     if (!ctx) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     const bool with_append = k_new != nullptr || v_new != nullptr;
@@ -311,7 +326,9 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         q_rows += ql;
     }
     int32_t n_units = 0, n_partials = 0;
-    if (plan_partition(n_req, ctx->kv_lens.data(), q_lens, ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, ctx->sm_count, ctx->tune,
+    PlanTuning tune = ctx->tune;
+    if (gs) tune.pool_pct = 0;  // (the pool's claim counter assumes one launch per plan, in plan order: a graph may be replayed at will)
+    if (plan_partition(n_req, ctx->kv_lens.data(), q_lens, ctx->cfg.n_q_heads, ctx->cfg.n_kv_heads, ctx->sm_count, tune,
                        ctx->items, ctx->cta_begin, &n_units, &n_partials, &ctx->plan_scratch, causal_tail) != 0)
         return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
     const int32_t n_items = (int32_t)ctx->items.size();
@@ -348,20 +365,24 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
             if (w.tile_end == (kv + XLLM_TILE_TOKENS - 1) / XLLM_TILE_TOKENS && (int64_t)w.tile_begin * XLLM_TILE_TOKENS > kv - ql) fuse = false;
         }
     }
+    if (with_append && !fuse && gs)
+        return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": this batch needs a separate append launch, whose parameters "
+                                                                   "change with the batch; append with xllm_kv_append outside the graph");
     if (with_append && !fuse) {  // two launches: the plan above already counts the new tokens
         const xllm_status as = xllm_kv_append(ctx, n_req, slots, q_lens ? q_lens : ctx->ones(n_req), k_new, v_new, cuda_stream);
         if (as != XLLM_OK) return as;
     }
 
-    int idx;
-    int e = acquire_stage(ctx, &idx);
+    int idx = -1;
+    int e = gs ? 0 : acquire_stage(ctx, &idx);
     if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
-    // staged blob: resolved items, then combine descriptors
-    const size_t off_items = 0;
+    // staged blob: (graph mode: the two launch records,) resolved items, then combine descriptors
+    const size_t off_al = 0, off_cl = align_up(sizeof(AttnLaunch), 16);
+    const size_t off_items = gs ? align_up(off_cl + sizeof(CombineLaunch), 16) : 0;
     const size_t off_comb = align_up(off_items + sizeof(DevItem) * (size_t)n_items, 16);
     const size_t total = align_up(off_comb + sizeof(CombineDesc) * combine.size(), 16);
-    if (total > ctx->stage_bytes) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
-    char *h = ctx->h_stage[idx];
+    if (total > (gs ? gs->bytes : ctx->stage_bytes)) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
+    char *h = gs ? gs->h_buf : ctx->h_stage[idx];
     DevItem *di = reinterpret_cast<DevItem *>(h + off_items);
     const int64_t head_tile = head_tile_bytes(ctx->cfg.head_dim);
     for (int32_t i = 0; i < n_items; ++i) {
@@ -388,7 +409,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    char *d = ctx->d_stage[idx];  // the same bytes seen from the device (mapped pinned memory)
+    char *d = gs ? gs->d_buf : ctx->d_stage[idx];  // the same bytes seen from the device (mapped pinned memory)
 
     AttnLaunch al{};
     al.items = reinterpret_cast<const DevItem *>(d + off_items);
@@ -414,20 +435,24 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     al.n_ctas = ctx->sm_count;
     al.debug_stall_cta = -1;
     std::memcpy(al.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
-    if (ctx->inject_timeouts > 0) {
+    if (ctx->inject_timeouts > 0 && !gs) {
         --ctx->inject_timeouts;
         for (int32_t c = 0; c < ctx->sm_count; ++c)
             if (al.cta_begin[c] < al.cta_begin[c + 1]) { al.debug_stall_cta = c; break; }
     }
     for (int32_t c = 0; c < ctx->sm_count; ++c)
         if (al.cta_begin[c] < al.cta_begin[c + 1]) al.first_item[c] = di[al.cta_begin[c]];
-    time_begin(ctx, 0, stream);
-    e = launch_attention(al, stream);
-    time_end(ctx, stream);
-    if (e) return cuda_fail(ctx, "launching the attention kernel", e);
-    if (al.n_pool > 0) ctx->pool_base += (uint32_t)al.n_pool + (uint32_t)al.n_ctas;  // every CTA's last claim fails, exactly once
-    ++ctx->st.kernel_launches;
-    if (!combine.empty()) {
+    if (!gs) {
+        time_begin(ctx, 0, stream);
+        e = launch_attention(al, stream);
+        time_end(ctx, stream);
+        if (e) return cuda_fail(ctx, "launching the attention kernel", e);
+        if (al.n_pool > 0) ctx->pool_base += (uint32_t)al.n_pool + (uint32_t)al.n_ctas;  // every CTA's last claim fails, exactly once
+        ++ctx->st.kernel_launches;
+    } else {
+        std::memcpy(h + off_al, &al, sizeof(al));
+    }
+    if (!combine.empty() || gs) {
         CombineLaunch cl{};
         cl.descs = reinterpret_cast<const CombineDesc *>(d + off_comb);
         cl.n_units = (int32_t)combine.size();
@@ -438,13 +463,20 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
         cl.n_q_heads = ctx->cfg.n_q_heads;
         cl.head_dim = ctx->cfg.head_dim;
         cl.out_f32 = out_f32 ? 1 : 0;
-        time_begin(ctx, 1, stream);
-        e = launch_combine(cl, stream);
-        time_end(ctx, stream);
-        if (e) return cuda_fail(ctx, "launching the combine kernel", e);
-        ++ctx->st.kernel_launches;
+        if (!gs) {
+            time_begin(ctx, 1, stream);
+            e = launch_combine(cl, stream);
+            time_end(ctx, stream);
+            if (e) return cuda_fail(ctx, "launching the combine kernel", e);
+            ++ctx->st.kernel_launches;
+        } else {
+            std::memcpy(h + off_cl, &cl, sizeof(cl));
+        }
     }
-    finish_launch(ctx, idx, stream);
+    if (gs)
+        gs->planned = true;
+    else
+        finish_launch(ctx, idx, stream);
     for (int32_t i = 0; i < n_req; ++i) {
         SlotRecord &s = ctx->xt->slot(slots[i]);
         s.last_use = ctx->seq;
@@ -591,6 +623,12 @@ xllm_status xllm_shutdown(xllm_ctx *ctx) {
         if (ctx->d_part_lse) cudaFree(ctx->d_part_lse);
         if (ctx->d_counters) cudaFree(ctx->d_counters);
         if (ctx->d_trace) cudaFree(ctx->d_trace);
+        for (GraphStep *gs : ctx->graph_steps)
+            if (gs) {
+                cudaFree(gs->d_cl);
+                cudaFreeHost(gs->h_buf);
+                delete gs;
+            }
         if (ctx->h_error) cudaFreeHost(ctx->h_error);
         for (TimedLaunch &t : ctx->timed) {
             cudaEventDestroy(t.start);
@@ -888,6 +926,74 @@ xllm_status xllm_append_verify_attention(xllm_ctx *ctx, int32_t n_req, const int
     if (ctx && (!q_lens || !k_new || !v_new))
         return fail(ctx, XLLM_ERR_INVALID, "append_verify_attention: q_lens, k_new and v_new must be non-null");
     return attention_impl(ctx, n_req, slots, q_lens, q, out, lse_out, scale, cuda_stream, "append_verify_attention", k_new, v_new);
+}
+
+xllm_status xllm_graph_step_create(xllm_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *out, float *lse_out,
+                                   float scale, int32_t *handle_out) {
+    if (!ctx || !handle_out) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "graph_step_create: context is host-only, no GPU work possible");
+    if (!q || !out || (k_new == nullptr) != (v_new == nullptr))
+        return fail(ctx, XLLM_ERR_INVALID, "graph_step_create: q and out must be non-null; k_new and v_new both or neither");
+    GraphStep *gs = new GraphStep();
+    gs->bytes = align_up(sizeof(AttnLaunch), 16) + align_up(sizeof(CombineLaunch), 16) +
+                align_up(sizeof(DevItem) * (size_t)ctx->max_items, 16) + align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16);
+    cudaError_t e = cudaHostAlloc(reinterpret_cast<void **>(&gs->h_buf), gs->bytes, cudaHostAllocMapped);
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&gs->d_buf), gs->h_buf, 0);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&gs->d_cl), sizeof(CombineLaunch));
+    if (e == cudaSuccess) e = cudaMemset(gs->d_cl, 0, sizeof(CombineLaunch));
+    if (e != cudaSuccess) {
+        if (gs->d_cl) cudaFree(gs->d_cl);
+        if (gs->h_buf) cudaFreeHost(gs->h_buf);
+        delete gs;
+        return cuda_fail(ctx, "graph_step_create: allocating the launch record", (int)e);
+    }
+    gs->q = q, gs->k_new = k_new, gs->v_new = v_new, gs->out = out, gs->lse_out = lse_out, gs->scale = scale;
+    ctx->graph_steps.push_back(gs);
+    *handle_out = (int32_t)ctx->graph_steps.size() - 1;
+    return XLLM_OK;
+}
+
+static GraphStep *graph_step_of(xllm_ctx *ctx, int32_t handle) {
+    return (handle >= 0 && (size_t)handle < ctx->graph_steps.size()) ? ctx->graph_steps[(size_t)handle] : nullptr;
+}
+
+xllm_status xllm_graph_step_plan(xllm_ctx *ctx, int32_t handle, int32_t n_req, const int32_t *slots, const int32_t *q_lens) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    GraphStep *gs = graph_step_of(ctx, handle);
+    if (!gs) return fail(ctx, XLLM_ERR_INVALID, "graph_step_plan: no such handle");
+    return attention_impl(ctx, n_req, slots, q_lens, gs->q, gs->out, gs->lse_out, gs->scale, nullptr, "graph_step_plan", gs->k_new,
+                          gs->v_new, nullptr, false, gs);
+}
+
+xllm_status xllm_graph_step_launch(xllm_ctx *ctx, int32_t handle, void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    GraphStep *gs = graph_step_of(ctx, handle);
+    if (!gs) return fail(ctx, XLLM_ERR_INVALID, "graph_step_launch: no such handle");
+    if (!gs->planned) return fail(ctx, XLLM_ERR_INVALID, "graph_step_launch: call xllm_graph_step_plan first");
+    int e = launch_attention_indirect(reinterpret_cast<const AttnLaunch *>(gs->d_buf),
+                                      reinterpret_cast<const CombineLaunch *>(gs->d_buf + align_up(sizeof(AttnLaunch), 16)), gs->d_cl,
+                                      ctx->cfg.head_dim, ctx->sm_count, cuda_stream);
+    if (e) return cuda_fail(ctx, "launching the attention kernel (graph mode)", e);
+    e = launch_combine_indirect(gs->d_cl, ctx->cfg.head_dim, ctx->sm_count, cuda_stream);
+    if (e) return cuda_fail(ctx, "launching the combine kernel (graph mode)", e);
+    ctx->st.kernel_launches += 2;
+    return XLLM_OK;
+}
+
+xllm_status xllm_graph_step_destroy(xllm_ctx *ctx, int32_t handle) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    GraphStep *gs = graph_step_of(ctx, handle);
+    if (!gs) return fail(ctx, XLLM_ERR_INVALID, "graph_step_destroy: no such handle");
+    cudaDeviceSynchronize();  // a replay may still be reading the record
+    cudaFree(gs->d_cl);
+    cudaFreeHost(gs->h_buf);
+    delete gs;
+    ctx->graph_steps[(size_t)handle] = nullptr;
+    return XLLM_OK;
 }
 
 xllm_status xllm_partial_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens,

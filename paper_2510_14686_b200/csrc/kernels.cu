@@ -67,7 +67,8 @@ struct Cfg {
     static constexpr int kOffQ = kOffP + 2 * 2 * kMaxRows * kPPitch;
     static constexpr int kOffItems = kOffQ + 2 * kMaxRows * kQPitch;
     static constexpr int kOffPool = kOffItems + kItemBatch * (int)sizeof(DevItem);   // [kPoolSlots] records claimed from the shared pool
-    static constexpr int kOffBars = kOffPool + kPoolSlots * (int)sizeof(DevItem);
+    static constexpr int kOffHeader = kOffPool + kPoolSlots * (int)sizeof(DevItem);  // graph mode: launch header, first record, own range
+    static constexpr int kOffBars = kOffHeader + (int)sizeof(AttnHeader) + (int)sizeof(DevItem) + 8;
     static constexpr int kNumBars = 2 * kHalfStages + 8 + 2 * kPoolSlots;
     static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast
     static constexpr int kSmemBytes = kOffFlags + 16;
@@ -336,7 +337,7 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
 // The caller fences (generic -> async proxy) and synchronises before the tiles are fetched.
 template <int D>
 __device__ __forceinline__ void append_new_rows(const DevItem *sitems, const DevItem &first, bool use_first, int nb,
-                                                const AttnLaunch &p, int64_t tile_block, int tid, int nthreads) {
+                                                const AttnHeader &p, int64_t tile_block, int tid, int nthreads) {
     constexpr int cpr = D / 8;  // 16-byte chunks per head row
     int max_new = 0;
     for (int i = 0; i < nb; ++i) max_new = max(max_new, (use_first && i == 0) ? first.n_new : sitems[i].n_new);
@@ -370,8 +371,10 @@ __device__ __forceinline__ void append_new_rows(const DevItem *sitems, const Dev
     }
 }
 
+// The whole kernel: `p` is the launch header (kernel parameters, or a copy in shared memory), [item_lo, item_hi) this
+// CTA's own run in p.items and `first_rec` a copy of its first record.
 template <int D, bool TRACE>
-__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnLaunch p) {
+__device__ __forceinline__ void attention_body(const AttnHeader &p, const int item_lo, const int item_hi, const DevItem &first_rec) {
     using C = Cfg<D>;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem_base = smem_u32(smem);
@@ -392,7 +395,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     const unsigned long long t_start = TRACE ? clock64() : 0ull;
     const unsigned long long g_start = TRACE ? globaltimer_ns() : 0ull;
 
-    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
     if (tid == 0) {
         for (int s = 0; s < C::kHalfStages; ++s) {
             mbar_init(bar_full + s * 8, 1);
@@ -454,7 +456,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 if (lane == 0) mbar_arrive(bar_items);
                 if (p.k_new) {  // fused append: these warps are idle until the first item finishes
                     mbar_wait(bar_items, 0, abort_flag, p.error_flag, 8);
-                    append_new_rows<D>(sitems, p.first_item[blockIdx.x], true, nb, p, (int64_t)p.n_kv_heads * 2 * C::kHalfTile,
+                    append_new_rows<D>(sitems, first_rec, true, nb, p, (int64_t)p.n_kv_heads * 2 * C::kHalfTile,
                                        tid - kEpilogueWarp0 * 32, kEpilogueThreads);
                     __threadfence();
                     asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores before the bulk copies that read them
@@ -478,7 +480,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         // record of item i of this batch; waits (once) for the fetch above before the first use of shared memory
         bool items_ready = !first_batch;
         auto item_at = [&](int i) -> DevItem {
-            if (first_batch && i == 0) return p.first_item[blockIdx.x];
+            if (first_batch && i == 0) return first_rec;
             if (!items_ready) {
                 mbar_wait(bar_items, 0, abort_flag, p.error_flag, 8);
                 items_ready = true;
@@ -899,9 +901,39 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     }
 }
 
+template <int D, bool TRACE>
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnLaunch p) {
+    attention_body<D, TRACE>(p, p.cta_begin[blockIdx.x], p.cta_begin[blockIdx.x + 1], p.first_item[blockIdx.x]);
+}
+
+// Graph mode: the same kernel with its launch record in memory (host memory mapped into the device, rewritten by the
+// host between replays of a captured graph), so that the kernel node's parameters never change.  Each CTA fetches the
+// header, its own range and its first record in one batch of loads.
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel_indirect(const AttnLaunch *rec, const CombineLaunch *cl_src,
+                                                                         CombineLaunch *cl_dst) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    // the second kernel's record goes to device memory here: its many small blocks then read it from L2, not over PCIe
+    if (blockIdx.x == 0 && threadIdx.x == kThreads - 1) *cl_dst = *cl_src;
+    constexpr int kHdrWords = (int)(sizeof(AttnHeader) / 4), kItemWords = (int)(sizeof(DevItem) / 4);
+    static_assert(sizeof(AttnHeader) % 8 == 0 && kHdrWords + kItemWords + 2 <= kThreads, "one word per thread");
+    uint32_t *dst = reinterpret_cast<uint32_t *>(smem + Cfg<D>::kOffHeader);
+    const int t = threadIdx.x;
+    if (t < kHdrWords)
+        dst[t] = reinterpret_cast<const uint32_t *>(static_cast<const AttnHeader *>(rec))[t];
+    else if (t < kHdrWords + kItemWords)
+        dst[t] = reinterpret_cast<const uint32_t *>(rec->first_item + blockIdx.x)[t - kHdrWords];
+    else if (t < kHdrWords + kItemWords + 2)
+        dst[t] = (uint32_t)rec->cta_begin[blockIdx.x + (t - kHdrWords - kItemWords)];
+    __syncthreads();
+    const AttnHeader &h = *reinterpret_cast<const AttnHeader *>(dst);
+    const DevItem &first = *reinterpret_cast<const DevItem *>(dst + kHdrWords);
+    attention_body<D, false>(h, (int)dst[kHdrWords + kItemWords], (int)dst[kHdrWords + kItemWords + 1], first);
+}
+
 // ---- LSE combine: merge the partial results of every split unit -------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
+__device__ __forceinline__ void combine_body(const CombineLaunch &p) {
     grid_launch_dependents();
     const CombineDesc d = p.descs[blockIdx.x];  // written by the host before the launch: fetched while the attention kernel drains
     grid_dependency_wait();                     // the partial results come from the attention kernel launched just before
@@ -946,6 +978,20 @@ __global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
     else
         static_cast<__nv_bfloat16 *>(p.out)[off * D + col] = __float2bfloat16_rn(res);
     if (col == 0 && p.lse_out) p.lse_out[off] = (W > 0.f) ? (M + log2f(W)) * 0.69314718055994531f : -INFINITY;
+}
+
+template <int D>
+__global__ void __launch_bounds__(D) combine_kernel(const CombineLaunch p) {
+    combine_body<D>(p);
+}
+
+// Graph mode: always launched, with a grid for the largest number of split units; the record (device memory, copied
+// there by the attention kernel before it) says how many there are this time.
+template <int D>
+__global__ void __launch_bounds__(D) combine_kernel_indirect(const CombineLaunch *rec) {
+    const CombineLaunch p = *rec;
+    if ((int)blockIdx.x >= p.n_units) return;
+    combine_body<D>(p);
 }
 
 // ---- merge of partial results computed over parts of longer sequences (possibly on other GPUs) --------------
@@ -1038,10 +1084,14 @@ int configure_kernels(int32_t head_dim) {
         e = cudaFuncSetAttribute(attention_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_kernel_indirect<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
     } else {
         e = cudaFuncSetAttribute(attention_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_kernel_indirect<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
     }
     return (int)e;
 }
@@ -1080,6 +1130,28 @@ int launch_combine(const CombineLaunch &p, void *stream) {
     dim3 grid(p.n_units, kMaxRows);
     if (p.head_dim == 128) return (int)launch_pdl(combine_kernel<128>, grid, dim3(128), 0, st, p);
     return (int)launch_pdl(combine_kernel<64>, grid, dim3(64), 0, st, p);
+}
+
+int launch_attention_indirect(const AttnLaunch *rec, const CombineLaunch *cl_src, CombineLaunch *cl_dst, int32_t head_dim,
+                              int32_t n_ctas, void *stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // plain launches: inside a captured graph the nodes are ordered by the graph (the kernels' dependency-control
+    // instructions do nothing without the launch attribute)
+    if (head_dim == 128)
+        attention_kernel_indirect<128><<<dim3(n_ctas), dim3(kThreads), Cfg<128>::kSmemBytes, st>>>(rec, cl_src, cl_dst);
+    else
+        attention_kernel_indirect<64><<<dim3(n_ctas), dim3(kThreads), Cfg<64>::kSmemBytes, st>>>(rec, cl_src, cl_dst);
+    return (int)cudaGetLastError();
+}
+
+int launch_combine_indirect(const CombineLaunch *rec, int32_t head_dim, int32_t max_units, void *stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 grid(max_units, kMaxRows);
+    if (head_dim == 128)
+        combine_kernel_indirect<128><<<grid, dim3(128), 0, st>>>(rec);
+    else
+        combine_kernel_indirect<64><<<grid, dim3(64), 0, st>>>(rec);
+    return (int)cudaGetLastError();
 }
 
 int launch_merge_parts(int32_t n_parts, int64_t rows, int32_t n_q_heads, int32_t head_dim, const float *out_parts,

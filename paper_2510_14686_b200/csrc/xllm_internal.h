@@ -118,7 +118,9 @@ struct AppendLaunch {
     AppendDesc d[kAppendBatch];
 };
 
-struct AttnLaunch {
+// What every CTA of an attention launch needs: travels in the kernel parameters, or (graph mode) sits in host memory
+// mapped into the device and is fetched by each CTA when it starts.
+struct AttnHeader {
     const DevItem *items;         // device, grouped by CTA
     const void *q;
     const void *k_new, *v_new;    // fused append: rows [sum n_new, H_kv, D] of the step's new tokens, else null
@@ -137,6 +139,9 @@ struct AttnLaunch {
     float scale_log2;             // scale * log2(e)
     int32_t n_ctas;
     int32_t debug_stall_cta;      // -1; else that CTA arms the V half of its first tile but never copies it (timeout test)
+};
+
+struct AttnLaunch : AttnHeader {
     int32_t cta_begin[kMaxCtas + 1];  // CTA c owns items [cta_begin[c], cta_begin[c+1])
     DevItem first_item[kMaxCtas];     // copy of items[cta_begin[c]]: the first loads need no trip to the item list
 };
@@ -158,6 +163,10 @@ constexpr int32_t kTraceWords = 16;  // per-CTA words of the optional trace buff
 int attention_smem_bytes(int32_t head_dim);
 int configure_kernels(int32_t head_dim);  // cudaFuncSetAttribute for the dynamic shared memory; returns cudaError
 int launch_attention(const AttnLaunch &p, void *stream);
+// graph mode: the launch records are read from (mapped host) memory by the kernels, so the launch parameters never change
+int launch_attention_indirect(const AttnLaunch *rec, const CombineLaunch *cl_src, CombineLaunch *cl_dst, int32_t head_dim,
+                              int32_t n_ctas, void *stream);
+int launch_combine_indirect(const CombineLaunch *rec, int32_t head_dim, int32_t max_units, void *stream);
 int launch_combine(const CombineLaunch &p, void *stream);
 int launch_merge_parts(int32_t n_parts, int64_t rows, int32_t n_q_heads, int32_t head_dim, const float *out_parts,
                        const float *lse_parts, void *out, float *lse_out, void *stream);

@@ -1,0 +1,110 @@
+"""GPU: graph mode.  A step is captured into a CUDA graph once; between replays only the launch record in mapped host
+memory is rewritten (other batch composition, other lengths, new rows appended) and every replay matches the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_14686_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+def test_one_capture_many_batches(binding):
+    import gpu_harness as gh
+
+    hq, hkv, d = 32, 8, 128
+    lens = [3000, 700, 65, 130, 5000, 64, 1, 2049]
+    batch = wl.custom_batch(801, hq, hkv, d, lens, [1] * len(lens))
+    s = batch.shape
+    max_rows = len(lens)
+    with gh.make_ctx(binding, s, len(lens), max(lens) + 64, [l + 64 for l in lens]) as ctx:
+        slots = gh.load_requests(ctx, batch.requests)
+        q = torch.zeros((max_rows, hq, d), dtype=torch.int16, device="cuda")
+        out = torch.zeros_like(q)
+        lse = torch.zeros((max_rows, hq), dtype=torch.float32, device="cuda")
+        h = ctx.graph_step_create(q, out, lse, scale=s.scale)
+        with pytest.raises(binding.XllmError):
+            ctx.graph_step_launch(h)                                   # nothing planned yet
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        ctx.graph_step_plan(h, slots)                                  # the record must exist when the kernels first run
+        with torch.cuda.stream(side):
+            ctx.graph_step_launch(h, side.cuda_stream)                 # warm-up outside capture (module load, attributes)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            ctx.graph_step_launch(h, torch.cuda.current_stream().cuda_stream)
+
+        def replay_and_check(sub):                                     # sub: indices of the requests in this batch
+            reqs = [batch.requests[i] for i in sub]
+            q[:len(sub)].copy_(gh.dev_bits(np.concatenate([r.q for r in reqs], axis=0)))
+            out.zero_()
+            ctx.graph_step_plan(h, [slots[i] for i in sub])
+            graph.replay()
+            torch.cuda.synchronize()
+            ctx.sync_check()
+            import oracle
+            o, l = oracle.attention_batch([r.q for r in reqs], [r.k[:r.kv_len] for r in reqs], [r.v[:r.kv_len] for r in reqs], s.scale)
+            gh.assert_parity(gh.host_bits(out[:len(sub)]), lse[:len(sub)].cpu().numpy(), np.concatenate(o), np.concatenate(l))
+
+        replay_and_check(list(range(len(lens))))                       # the captured batch
+        replay_and_check([4, 0, 7])                                    # fewer requests, another order
+        replay_and_check([6])                                          # one request of one token
+        # shorter contexts: roll three slots back, then the same graph again
+        for i, new_len in ((0, 1000), (4, 64), (1, 699)):
+            ctx.kv_set_len(slots[i], new_len)
+            batch.requests[i].kv_len = new_len
+        replay_and_check(list(range(len(lens))))
+        ctx.graph_step_destroy(h)
+        with pytest.raises(binding.XllmError):
+            ctx.graph_step_plan(h, slots)
+
+
+def test_captured_step_with_fused_append(binding):
+    """k_new / v_new bound: every replay appends the step's rows and attends over the grown contexts."""
+    import gpu_harness as gh
+    import oracle
+
+    hq, hkv, d = 28, 4, 128
+    lens = [900, 64, 63, 2500, 128]
+    steps = 3
+    batch = wl.custom_batch(802, hq, hkv, d, [l + steps for l in lens], [1] * len(lens))
+    s = batch.shape
+    n = len(lens)
+    with gh.make_ctx(binding, s, n, max(lens) + 64, [l + 64 for l in lens]) as ctx:
+        slots = []
+        for r, l in zip(batch.requests, lens):
+            sl = ctx.kv_reserve(expected_tokens=l + steps)
+            ctx.kv_map_pages(sl, l + steps)
+            ctx.kv_append([sl], [l], gh.dev_bits(r.k[:l]), gh.dev_bits(r.v[:l]))
+            slots.append(sl)
+        q = gh.dev_bits(np.concatenate([r.q for r in batch.requests], axis=0))
+        k_new = torch.zeros((n, hkv, d), dtype=torch.int16, device="cuda")
+        v_new = torch.zeros_like(k_new)
+        out = torch.zeros_like(q)
+        lse = torch.zeros((n, hq), dtype=torch.float32, device="cuda")
+        h = ctx.graph_step_create(q, out, lse, k_new, v_new, scale=s.scale)
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        for t in range(steps):
+            k_new.copy_(gh.dev_bits(np.stack([r.k[l + t] for r, l in zip(batch.requests, lens)])))
+            v_new.copy_(gh.dev_bits(np.stack([r.v[l + t] for r, l in zip(batch.requests, lens)])))
+            torch.cuda.synchronize()
+            ctx.graph_step_plan(h, slots)
+            if t == 0:
+                with torch.cuda.graph(graph, stream=side):
+                    ctx.graph_step_launch(h, torch.cuda.current_stream().cuda_stream)
+            graph.replay()
+            torch.cuda.synchronize()
+            ctx.sync_check()
+            o, l_ = oracle.attention_batch([r.q for r in batch.requests], [r.k[:l + t + 1] for r, l in zip(batch.requests, lens)],
+                                           [r.v[:l + t + 1] for r, l in zip(batch.requests, lens)], s.scale)
+            gh.assert_parity(gh.host_bits(out), lse.cpu().numpy(), np.concatenate(o), np.concatenate(l_))
+            for sl, l in zip(slots, lens):
+                assert ctx.kv_slot_info(sl).kv_len == l + t + 1

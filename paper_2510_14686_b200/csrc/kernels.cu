@@ -500,21 +500,6 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
 
         if (warp == kProducerWarp) {
             // ================= producer =================
-            union Record {
-                DevItem it;
-                uint4 w[3];
-            } next;  // pool: the record just claimed
-            bool have = false;
-            auto claim = [&]() {  // one more record of the pool, or none: every CTA's last claim fails, exactly once
-                const uint32_t t = atomicAdd(p.pool_counter, 1u) - p.pool_base;
-                have = t < (uint32_t)p.n_pool;
-                if (have) {       // (host memory: the latency overlaps with the copies issued in the meantime)
-                    const uint4 *src = reinterpret_cast<const uint4 *>(p.items + p.pool_first + t);
-                    next.w[0] = src[0];
-                    next.w[1] = src[1];
-                    next.w[2] = src[2];
-                }
-            };
             // One elected lane issues every copy.  In the pool segment the other lanes follow it item by item, because an
             // item that carries new K/V rows (a whole unit, in a launch that appends) has them written by this warp first.
             for (int i = 0; i < nb && (pool || lane == 0); ++i) {
@@ -525,18 +510,24 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
                     const uint32_t ps = i % kPoolSlots, pph = (i / kPoolSlots) & 1;
                     int go = 0;
                     if (lane == 0) {
-                        // Claimed only now, when this CTA is ready to issue it: a CTA that claimed ahead would take work
-                        // from one that is further along.  (The record comes from host memory; the tiles already in the
-                        // ring cover most of that latency.)
-                        claim();
+                        // One more record of the pool, or none (every CTA's last claim fails, exactly once).  Claimed only
+                        // now, when this CTA is ready to issue it: a CTA that claimed ahead would take work from one that is
+                        // further along.  The record comes from host memory straight into the slot; the tiles already in
+                        // the ring cover most of that latency.
+                        const uint32_t t = atomicAdd(p.pool_counter, 1u) - p.pool_base;
+                        const bool have = t < (uint32_t)p.n_pool;
                         const bool ok = mbar_wait(bar_pempty + ps * 8, pph ^ 1, abort_flag, p.error_flag, 11);
-                        Record pub = next;
-                        if (!have) pub.it.tile_begin = pub.it.tile_end = -1;  // end of the pool
                         if (ok) {
                             uint4 *dst = reinterpret_cast<uint4 *>(smem + C::kOffPool) + ps * 3;
-                            dst[0] = pub.w[0];
-                            dst[1] = pub.w[1];
-                            dst[2] = pub.w[2];
+                            if (have) {
+                                const uint4 *src = reinterpret_cast<const uint4 *>(p.items + p.pool_first + t);
+                                const uint4 w0 = src[0], w1 = src[1], w2 = src[2];
+                                dst[0] = w0;
+                                dst[1] = w1;
+                                dst[2] = w2;
+                            } else {
+                                dst[1] = make_uint4(0xffffffffu, 0xffffffffu, 0u, 0u);  // tile_begin = tile_end = -1: end of the pool
+                            }
                             mbar_arrive(bar_pfull + ps * 8);
                         }
                         go = have && ok;

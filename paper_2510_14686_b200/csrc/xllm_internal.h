@@ -23,7 +23,7 @@ struct PlanTuning {
     // several percent in the bandwidth they get).  0: no pool.  Measured on B200: 6 is best on the speculative-
     // verification batch; batches of many short requests gain up to 15.
     int32_t pool_pct = 8;
-    int32_t pool_min_tiles = 4;   // units smaller than this stay with a CTA: claiming costs about as much as they do
+    int32_t pool_min_tiles = 2;   // single-tile units stay with a CTA: claiming one costs about as much as it does (2 measured better than 4)
     int32_t pool_share_div = 8;   // ... and units larger than a CTA's share / this are too coarse to even anything out
 };
 

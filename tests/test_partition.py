@@ -42,7 +42,7 @@ def check_plan(binding, kv, ql, hq, hkv, n_ctas):
             if c < n_ctas:
                 loads[c] += cost + 6 + 8 * it.n_q_tok * it.n_g // 16   # every piece pays the unit's fixed cost
             else:
-                assert it.partial_idx < 0 and it.tile_begin == 0 and it.tile_end == nt and 4 <= nt <= 64   # whole small units only
+                assert it.partial_idx < 0 and it.tile_begin == 0 and it.tile_end == nt and 2 <= nt <= 64   # whole small units only
             key = (it.req, it.kv_head, it.q_tok0, it.g0)
             q_len = 1 if ql is None else int(ql[it.req])
             vis_last = int(kv[it.req]) - q_len + it.q_tok0 + it.n_q_tok

@@ -54,7 +54,10 @@ struct Cfg {
         slot = (g ? kSlotsA : 0) + hl % n;
         phase = (hl / n) & 1;
     }
-    static constexpr int kQPitch = D * 2 + 16;                       // bytes, padded against bank conflicts
+    // bytes per query row: padded by one 16-byte chunk.  Not only against bank conflicts of the fragment loads: with a pitch
+    // that is a multiple of 128 bytes (dense rows, or padded by 128) sporadic wrong query rows were measured on short items,
+    // with pitches of 272, 288 and 320 bytes never; the cause was not found, so the rows stay padded and copied one by one.
+    static constexpr int kQPitch = D * 2 + 16;
     static constexpr int kOPitch = D + 8;                            // floats
     static constexpr int kPPitch = T * 2 + 16;                       // bytes per row of the bf16 weight tile
     static constexpr int kColsPerWarp = D / 4;                       // head-dim columns a warp accumulates
@@ -92,6 +95,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // back: those reads have completed before the arrival is issued.
 __device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar, float after) {
     asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];  // %1" ::"r"(bar), "f"(after) : "memory");
+}
+// A releasing arrival that is issued only after `after` (a value computed from registers that loads filled) is available.
+__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, uint32_t after) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // %1" ::"r"(bar), "r"(after) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -624,8 +631,15 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
                         if (g8 + 8 >= n_rows) qf[ks][1] = qf[ks][3] = 0u;
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_qempty + qb * 8);
+                {
+                    // The buffer goes back to the producer only when the fragment loads above have delivered: nothing else
+                    // before the arrival depends on them, and a load still in flight would see the next item's rows.
+                    uint32_t dep = 0;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) dep ^= qf[ks][0] ^ qf[ks][1] ^ qf[ks][2] ^ qf[ks][3];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_after(bar_qempty + qb * 8, dep);
+                }
 
                 const int limit_lo = (g8 < n_rows) ? row_limit0 + (all_visible ? 0 : g8 / it.n_g) : 0;
                 const int limit_hi = (g8 + 8 < n_rows) ? row_limit0 + (all_visible ? 0 : (g8 + 8) / it.n_g) : 0;

@@ -108,6 +108,27 @@ def test_verify_mixed_q_lens_and_causal_mask(binding, hq, hkv, d, maxq):
     # bitwise equality is not required (different work split), agreement within the edge bound is.
 
 
+def test_many_short_items_repeatedly(binding):
+    """Short requests fly through a CTA in a few hundred nanoseconds each, which is where buffer hand-offs between the
+    producer, the consumers and the epilogue are under the most pressure: many launches, every one against the oracle."""
+    import gpu_harness as gh
+
+    rng = np.random.default_rng(99)
+    lens, qls = [], []
+    for _ in range(160):
+        ql = int(rng.integers(1, 5))
+        lens.append(int(rng.integers(ql, 140)))
+        qls.append(ql)
+    batch = wl.custom_batch(901, 32, 8, 128, lens, qls)
+    with gh.make_ctx(binding, batch.shape, len(lens), max(lens) + 8, lens, max_q_len=4) as ctx:
+        slots = gh.load_requests(ctx, batch.requests)
+        first, first_lse = gh.run_attention(ctx, batch, slots)
+        check_edge(first, first_lse, batch)
+        for _ in range(15):
+            out, lse = gh.run_attention(ctx, batch, slots)
+            assert np.array_equal(out, first) and np.array_equal(lse, first_lse)
+
+
 def test_verify_rows_match_decode_on_truncated_context(binding):
     import gpu_harness as gh
 

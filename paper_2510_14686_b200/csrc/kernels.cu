@@ -500,7 +500,8 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
             if (!__all_sync(0xffffffffu, mbar_wait(bar_pfull + ps * 8, pph, abort_flag, p.error_flag, 10))) return false;
             it = pool_items[ps];
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pempty + ps * 8);
+            // (the slot goes back only when the loads of the record have delivered: a field of each 16-byte piece)
+            if (lane == 0) mbar_arrive_after(bar_pempty + ps * 8, (uint32_t)it.q_row ^ (uint32_t)it.tile_begin ^ (uint32_t)it.n_new);
             return it.tile_begin >= 0;
         };
         int n_done = 0;  // items of this segment (the same in every warp)

@@ -54,9 +54,9 @@ struct Cfg {
         slot = (g ? kSlotsA : 0) + hl % n;
         phase = (hl / n) & 1;
     }
-    // bytes per query row: padded by one 16-byte chunk.  Not only against bank conflicts of the fragment loads: with a pitch
-    // that is a multiple of 128 bytes (dense rows, or padded by 128) sporadic wrong query rows were measured on short items,
-    // with pitches of 272, 288 and 320 bytes never; the cause was not found, so the rows stay padded and copied one by one.
+    // bytes per query row: padded by one 16-byte chunk against bank conflicts of the fragment loads.  (Dense rows would let
+    // the heads of one query token land with one copy, but the 8-way conflicts then cost about 1 us of shared-memory pipe
+    // per item: measured 4 % slower on decode, 17 % on batches of short requests.)
     static constexpr int kQPitch = D * 2 + 16;
     static constexpr int kOPitch = D + 8;                            // floats
     static constexpr int kPPitch = T * 2 + 16;                       // bytes per row of the bf16 weight tile
@@ -73,8 +73,8 @@ struct Cfg {
     static constexpr int kOffHeader = kOffPool + kPoolSlots * (int)sizeof(DevItem);  // graph mode: launch header, first record, own range
     static constexpr int kOffBars = kOffHeader + (int)sizeof(AttnHeader) + (int)sizeof(DevItem) + 8;
     static constexpr int kNumBars = 2 * kHalfStages + 8 + 2 * kPoolSlots;
-    static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast
-    static constexpr int kSmemBytes = kOffFlags + 16;
+    static constexpr int kOffFlags = kOffBars + kNumBars * 8;        // [0] abort flag, [1] arrival-count broadcast, [4..15] a scratch word per warp
+    static constexpr int kSmemBytes = kOffFlags + 64;
     static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
 
@@ -90,15 +90,19 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Arrival without release semantics, for a thread that has global stores in flight (a releasing arrive may first wait
-// until those are performed).  `after` is a value computed from everything the thread read from the buffer it hands
-// back: those reads have completed before the arrival is issued.
-__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar, float after) {
-    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];  // %1" ::"r"(bar), "f"(after) : "memory");
+// Hand-off of a buffer whose contents this thread has just loaded into registers: the arrival must not be issued before
+// the loads have delivered (a load still in flight would see what the other side writes next).  `after` is a value
+// computed from everything that was loaded; it is stored to a scratch word of shared memory first -- a real use, which
+// neither compiler nor assembler can drop, and which cannot issue before its operand exists -- and the arrival follows
+// in program order.  (An operand that only appears in a comment of the asm text is removed by the assembler.)
+__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, uint32_t after, uint32_t scratch) {
+    asm volatile("st.shared.b32 [%2], %1;\n\tmbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar), "r"(after), "r"(scratch) : "memory");
 }
-// A releasing arrival that is issued only after `after` (a value computed from registers that loads filled) is available.
-__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, uint32_t after) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // %1" ::"r"(bar), "r"(after) : "memory");
+// The same without release semantics, for a thread that has global stores in flight (a releasing arrive may first wait
+// until those are performed).
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar, float after, uint32_t scratch) {
+    asm volatile("st.shared.f32 [%2], %1;\n\tmbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar), "f"(after), "r"(scratch)
+                 : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -388,6 +392,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const DevItem *sitems = reinterpret_cast<const DevItem *>(smem + C::kOffItems);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::kOffFlags);
+    const uint32_t scratch_word = smem_base + C::kOffFlags + 16 + warp * 4;  // write-only sink of mbar_arrive_after
     const uint32_t bar_full = smem_base + C::kOffBars;               // [kHalfStages] K or V half of a tile landed
     const uint32_t bar_empty = bar_full + C::kHalfStages * 8;         // [kHalfStages] ... consumed (4 warps)
     const uint32_t bar_qfull = bar_empty + C::kHalfStages * 8;        // [2] query rows landed
@@ -501,7 +506,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
             it = pool_items[ps];
             __syncwarp();
             // (the slot goes back only when the loads of the record have delivered: a field of each 16-byte piece)
-            if (lane == 0) mbar_arrive_after(bar_pempty + ps * 8, (uint32_t)it.q_row ^ (uint32_t)it.tile_begin ^ (uint32_t)it.n_new);
+            if (lane == 0) mbar_arrive_after(bar_pempty + ps * 8, (uint32_t)it.q_row ^ (uint32_t)it.tile_begin ^ (uint32_t)it.n_new, scratch_word);
             return it.tile_begin >= 0;
         };
         int n_done = 0;  // items of this segment (the same in every warp)
@@ -639,7 +644,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) dep ^= qf[ks][0] ^ qf[ks][1] ^ qf[ks][2] ^ qf[ks][3];
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_after(bar_qempty + qb * 8, dep);
+                    if (lane == 0) mbar_arrive_after(bar_qempty + qb * 8, dep, scratch_word);
                 }
 
                 const int limit_lo = (g8 < n_rows) ? row_limit0 + (all_visible ? 0 : g8 / it.n_g) : 0;
@@ -760,7 +765,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
                 const int n_iter = (n_elems - (et & ~31) + kEpilogueThreads - 1) / kEpilogueThreads;  // (the same for the whole warp)
                 if (n_iter <= 0) {
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_relaxed(bar_mempty, 0.f);
+                    if (lane == 0) mbar_arrive_relaxed(bar_mempty, 0.f, scratch_word);
                 }
 #pragma unroll 1
                 for (int j = 0; j < n_iter; ++j) {
@@ -777,7 +782,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
                     }
                     if (j == n_iter - 1) {  // (n_iter is the same for the whole warp)
                         const float seen = acc.x + __shfl_xor_sync(0xffffffffu, acc.x, 1);  // every lane's loads have been used
-                        if (lane == 0) mbar_arrive_relaxed(bar_mempty, seen);
+                        if (lane == 0) mbar_arrive_relaxed(bar_mempty, seen, scratch_word);
                     }
                     if (!valid) continue;
                     if (it.partial_idx >= 0) {

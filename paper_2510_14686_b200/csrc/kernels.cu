@@ -123,10 +123,9 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // Bounded wait: gives up after kWaitLimitNs or as soon as another warp of the CTA gave up.  On failure the
 // CTA-wide abort flag (shared) and the host-visible error word are set and false is returned; callers then
 // skip their work but keep executing the barrier protocol so that no warp is left waiting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag,
-                                          int code) {
-    if (*abort_flag) return false;
-    if (mbar_try_wait(bar, parity)) return true;
+// (the waiting loop is kept out of line: the kernel has some twenty waits, most of them in its hottest loops, and the
+// instruction cache is a scarce resource here)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
@@ -139,6 +138,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag,
+                                          int code) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, error_flag, code);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -160,6 +165,13 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// 2^x by the hardware approximation (relative error about 2^-22, far below the bf16 rounding of what it feeds; inputs here
+// are <= 0 or -inf, results in [0, 1]): one instruction instead of the library routine's range handling, in the hottest loop.
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -257,14 +269,14 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
     mx0 = fmaxf(fmaxf(mxs[g8], mxs[kMaxRows + g8]), fmaxf(mxs[2 * kMaxRows + g8], mxs[3 * kMaxRows + g8]));
     const float mn0 = fmaxf(m[0], mx0 * scale_log2);
     const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0;
-    const float a0 = exp2f(m[0] - ms0);
+    const float a0 = fast_exp2(m[0] - ms0);
     m[0] = mn0;
     float ms1 = 0.f, a1 = 1.f;
     if (!HALF) {
         mx1 = fmaxf(fmaxf(mxs[g8 + 8], mxs[kMaxRows + g8 + 8]), fmaxf(mxs[2 * kMaxRows + g8 + 8], mxs[3 * kMaxRows + g8 + 8]));
         const float mn1 = fmaxf(m[1], mx1 * scale_log2);
         ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        a1 = exp2f(m[1] - ms1);
+        a1 = fast_exp2(m[1] - ms1);
         m[1] = mn1;
     }
     l[0] *= a0;
@@ -273,10 +285,10 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
         float p[2][4];
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
-            p[nt][0] = exp2f(fmaf(s[nt][0], scale_log2, -ms0));
-            p[nt][1] = exp2f(fmaf(s[nt][1], scale_log2, -ms0));
-            p[nt][2] = HALF ? 0.f : exp2f(fmaf(s[nt][2], scale_log2, -ms1));
-            p[nt][3] = HALF ? 0.f : exp2f(fmaf(s[nt][3], scale_log2, -ms1));
+            p[nt][0] = fast_exp2(fmaf(s[nt][0], scale_log2, -ms0));
+            p[nt][1] = fast_exp2(fmaf(s[nt][1], scale_log2, -ms0));
+            p[nt][2] = HALF ? 0.f : fast_exp2(fmaf(s[nt][2], scale_log2, -ms1));
+            p[nt][3] = HALF ? 0.f : fast_exp2(fmaf(s[nt][3], scale_log2, -ms1));
         }
         l[0] += (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
         if (!HALF) l[1] += (p[0][2] + p[0][3]) + (p[1][2] + p[1][3]);

@@ -358,8 +358,9 @@ __device__ __forceinline__ void consume_tile(uint32_t kstage, uint32_t vstage, u
 // All items of a batch are handled in one flat loop (item, 16-byte chunk) whose loads are issued four at a time before
 // their stores: the copy is a chain of HBM round trips otherwise.  `tid`/`nthreads`: the threads sharing the copy.
 // The caller fences (generic -> async proxy) and synchronises before the tiles are fetched.
+// (out of line: three call sites, 13 KB each when inlined, none of them hot -- the kernel's hot loops are faster with less code around them)
 template <int D>
-__device__ __forceinline__ void append_new_rows(const DevItem *sitems, const DevItem &first, bool use_first, int nb,
+__device__ __noinline__ void append_new_rows(const DevItem *sitems, const DevItem &first, bool use_first, int nb,
                                                 const AttnHeader &p, int64_t tile_block, int tid, int nthreads) {
     constexpr int cpr = D / 8;  // 16-byte chunks per head row
     int max_new = 0;

@@ -7,7 +7,10 @@
  *
  * Conventions for every call
  *   - "host" / "device" says where a pointer must live.  Device pointers belong to the caller
- *     (typically torch tensors); the library never frees them.
+ *     (typically torch tensors); the library never frees them.  A "device" tensor of a call (q, k_new,
+ *     v_new, out, lse_out, ...) may also be pinned host memory that the device can address (cudaHostAlloc,
+ *     cudaHostRegister; with unified addressing the same pointer): the kernels then fetch it and write it
+ *     over PCIe themselves, which saves the separate copies of a step whose inputs start on the host.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All
  *     kernels are launched on it; no call synchronises the stream unless stated.
  *   - Small host arrays (`slots`, `n_new`, `q_lens`) are consumed before the call returns.

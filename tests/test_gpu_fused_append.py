@@ -140,6 +140,34 @@ def test_fused_append_with_items_from_the_shared_pool(binding):
     gh.assert_parity(out, lse, *gh.oracle_batch(batch))
 
 
+def test_pinned_host_buffers_as_call_tensors(binding):
+    """q, k_new, v_new, out and lse_out in pinned host memory: the kernels reach them over PCIe; same bits as from HBM."""
+    import gpu_harness as gh
+
+    batch = wl.custom_batch(416, 28, 4, 128, [900, 64, 2100, 5, 130, 3000], [1] * 6)
+    out_dev, lse_dev, _ = run_fused(binding, batch)
+    s = batch.shape
+    lens = [r.kv_len for r in batch.requests]
+    with gh.make_ctx(binding, s, len(lens), max(lens) + 8, lens) as ctx:
+        slots = []
+        for r in batch.requests:
+            sl = ctx.kv_reserve(expected_tokens=r.kv_len)
+            ctx.kv_map_pages(sl, r.kv_len)
+            pre = r.kv_len - r.q_len
+            if pre:
+                ctx.kv_append([sl], [pre], gh.dev_bits(r.k[:pre]), gh.dev_bits(r.v[:pre]))
+            slots.append(sl)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        q = pin(np.concatenate([r.q for r in batch.requests]))
+        k_new = pin(np.concatenate([r.k[r.kv_len - r.q_len:] for r in batch.requests]))
+        v_new = pin(np.concatenate([r.v[r.kv_len - r.q_len:] for r in batch.requests]))
+        out = torch.zeros_like(q).pin_memory()
+        lse = torch.zeros(q.shape[:2], dtype=torch.float32).pin_memory()
+        ctx.append_decode_attention(slots, k_new, v_new, q, out, lse, s.scale)
+        ctx.sync_check()
+        assert np.array_equal(out.numpy().view(np.uint16), out_dev) and np.array_equal(lse.numpy(), lse_dev)
+
+
 def test_not_mapped_is_refused_before_anything_runs(binding):
     import gpu_harness as gh
 

@@ -187,3 +187,25 @@ def test_shutdown_with_jobs_pending_does_not_hang(binding):
     for r in range(20):
         ctx.kv_premap_async(slots, [400 * (r + 1)] * 6)
     ctx.shutdown()
+
+
+def test_host_only_context_refuses_every_kernel_launching_call(binding):
+    """The page bookkeeping runs without a GPU; everything that would launch a kernel says so instead of pretending."""
+    ctx, _ = make(binding)
+    with ctx:
+        s = ctx.kv_reserve(expected_tokens=100)
+        ctx.kv_map_pages(s, 100)
+        dummy = np.zeros(16, np.int16)      # never touched: the calls are refused before any pointer is used
+        calls = [
+            lambda: ctx.kv_append([s], [1], dummy, dummy, 0),
+            lambda: ctx.decode_attention([s], dummy, dummy, None, 1.0, 0),
+            lambda: ctx.verify_attention([s], [1], dummy, dummy, None, 1.0, 0),
+            lambda: ctx.append_decode_attention([s], dummy, dummy, dummy, dummy, None, 1.0, 0),
+            lambda: ctx.partial_attention([s], [1], [1], dummy, dummy.view(np.float32), dummy.view(np.float32), 1.0, 0),
+            lambda: ctx.graph_step_create(dummy, dummy),
+        ]
+        for call in calls:
+            with pytest.raises(binding.XllmError) as e:
+                call()
+            assert e.value.status == binding.ERR_UNSUPPORTED, str(e.value)
+        assert ctx.kv_slot_info(s).kv_len == 0

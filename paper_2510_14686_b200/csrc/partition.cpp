@@ -71,6 +71,19 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
         PlanUnit *begin() { return p; }
         PlanUnit *end() { return p + n; }
     } units{buf.units, 0, buf.cap_units, false};
+    // One pass builds the units with their costs (a full tile costs tile_cost; the last tile of a unit is fetched in
+    // 16-token steps: half of its cost is fixed, half goes with the volume; a unit's fixed cost grows with its row
+    // count), the total number of tiles and a histogram of the small units' sizes for the pool below.
+    constexpr int32_t kMaxWhole = 64;
+    int32_t hist[kMaxWhole + 1] = {0};
+    int64_t total_tiles = 0;
+    auto finish = [&](Unit &u, int64_t vis_last) {
+        const int32_t tail_rows = (int32_t)std::min<int64_t>(T, ((vis_last - (int64_t)(u.n_tiles - 1) * T) + 15) / 16 * 16);
+        u.last_cost = tune.tile_cost / 2 + tune.tile_cost * tail_rows / (2 * T);  // half fixed, half by volume
+        u.overhead = tune.unit_overhead + tune.row_overhead * u.n_q_tok * u.n_g / kMaxRows;
+        total_tiles += u.n_tiles;
+        if (u.n_tiles <= kMaxWhole) ++hist[u.n_tiles];
+    };
     for (int32_t r = 0; r < n_req; ++r) {
         const int64_t kv = kv_lens[r];
         const int32_t ql = q_lens ? q_lens[r] : 1;
@@ -85,6 +98,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
                     const int64_t vis_first = tail ? kv - ql + t0 + 1 : kv;  // keys visible to the first row
                     Unit u{r, h, (int16_t)t0, (int16_t)nt, 0, (int16_t)G, (int32_t)((vis_last + T - 1) / T),
                            (int32_t)((vis_first - 1) / T), 0, 0, 0};
+                    finish(u, vis_last);
                     units.push_back(u);
                 }
             } else {
@@ -93,6 +107,7 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
                     for (int32_t g0 = 0; g0 < G; g0 += kMaxRows) {
                         Unit u{r, h, (int16_t)t0, 1, (int16_t)g0, (int16_t)std::min(kMaxRows, G - g0),
                                (int32_t)((vis + T - 1) / T), (int32_t)((vis - 1) / T), 0, 0, 0};
+                        finish(u, vis);
                         units.push_back(u);
                     }
                 }
@@ -101,7 +116,6 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     }
     if (units.overflow) return -2;
     const int32_t U = static_cast<int32_t>(units.size());
-    int64_t *start = buf.start;
     int32_t *cta_begin = buf.cta_begin;
     struct ItemList {
         xllm_work_item *p;
@@ -117,49 +131,40 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     // without such units (a few very long sequences; or so little work that a CTA's run is a few tiles) gets no pool.
     // The pool is capped at kPoolMaxPerCta items per CTA: what it has to absorb grows with the run time of a CTA, not
     // with the batch.
+    int32_t quota[kMaxWhole + 1] = {0};  // units of each size that go to the pool
+    int32_t lo = 1, hi = 0;
+    int64_t got_items = 0;
     {
-        int64_t total_tiles = 0;
-        for (int32_t u = 0; u < U; ++u) total_tiles += units[u].n_tiles;
         const int64_t share = total_tiles / n_ctas;
         int64_t target_tiles = tune.pool_pct > 0 ? total_tiles * tune.pool_pct / 100 : 0;
         if (total_tiles < 8 * (int64_t)n_ctas) target_tiles = 0;
         const int64_t max_items = (int64_t)kPoolMaxPerCta * n_ctas;
-        constexpr int32_t kMaxWhole = 64;
-        const int32_t lo = std::max(1, tune.pool_min_tiles);
-        const int32_t hi = (int32_t)std::min<int64_t>(kMaxWhole, share / std::max(1, tune.pool_share_div));  // (much shorter than a CTA's run)
-        int32_t quota[kMaxWhole + 1] = {0};  // units of each size: first how many there are, then how many go to the pool
-        for (int32_t u = 0; u < U && target_tiles > 0; ++u)
-            if (units[u].n_tiles >= lo && units[u].n_tiles <= hi) ++quota[units[u].n_tiles];
-        int64_t got_tiles = 0, got_items = 0;
-        for (int32_t n = lo; n <= kMaxWhole; ++n) {  // smallest first, up to the target
+        lo = std::max(1, tune.pool_min_tiles);
+        hi = target_tiles > 0 ? (int32_t)std::min<int64_t>(kMaxWhole, share / std::max(1, tune.pool_share_div)) : 0;  // (much shorter than a CTA's run)
+        int64_t got_tiles = 0;
+        for (int32_t n = lo; n <= hi; ++n) {  // smallest first, up to the target
             const int64_t room_tiles = target_tiles - got_tiles, room_items = max_items - got_items;
-            const int64_t take = (n > hi || room_tiles <= 0 || room_items <= 0)
-                                     ? 0
-                                     : std::min<int64_t>(std::min<int64_t>(quota[n], (room_tiles + n - 1) / n), room_items);
+            if (room_tiles <= 0 || room_items <= 0) break;
+            const int64_t take = std::min<int64_t>(std::min<int64_t>(hist[n], (room_tiles + n - 1) / n), room_items);
             quota[n] = (int32_t)take;
             got_tiles += take * n;
             got_items += take;
         }
-        for (int32_t u = 0; u < U && got_items > 0; ++u) {
-            Unit &un = units[u];
-            if (un.n_tiles >= lo && un.n_tiles <= hi && quota[un.n_tiles] > 0) {
-                --quota[un.n_tiles];
-                un.pool_whole = 1;
-            }
-        }
     }
-    // cost axis: start position of every unit.  A full tile costs tile_cost; the last tile of a unit is fetched
-    // in 16-token steps: half of its cost is fixed, half goes with the volume; a unit's fixed cost grows with its row count.
+    // One pass: mark the pool's units and lay the others out on the cost axis.
+    int64_t *start = buf.start;
+    int64_t mean_overhead = 0;
     start[0] = 0;
     for (int32_t u = 0; u < U; ++u) {
         Unit &un = units[u];
-        const int64_t vis_last = (!causal_tail || causal_tail[un.req]) ? kv_lens[un.req] - (q_lens ? q_lens[un.req] : 1) + un.q_tok0 + un.n_q_tok
-                                                                      : kv_lens[un.req];
-        const int32_t tail_rows = (int32_t)std::min<int64_t>(T, ((vis_last - (int64_t)(un.n_tiles - 1) * T) + 15) / 16 * 16);
-        un.last_cost = tune.tile_cost / 2 + tune.tile_cost * tail_rows / (2 * T);  // half fixed, half by volume
-        un.overhead = tune.unit_overhead + tune.row_overhead * un.n_q_tok * un.n_g / kMaxRows;
+        if (got_items > 0 && un.n_tiles >= lo && un.n_tiles <= hi && quota[un.n_tiles] > 0) {
+            --quota[un.n_tiles];
+            un.pool_whole = 1;
+        }
+        mean_overhead += un.overhead;
         start[u + 1] = start[u] + (un.pool_whole ? 0 : un.overhead + (int64_t)tune.tile_cost * (un.n_tiles - 1) + un.last_cost);
     }
+    mean_overhead = U ? mean_overhead / U : 0;
     // Walk the axis once, CTA by CTA.  Each CTA aims at an equal share of what is still to be done; "what is
     // still to be done" includes the fixed cost a unit's continuation pays again when a cut splits the unit, so the
     // shares stay equal although every split adds work.
@@ -167,9 +172,6 @@ int plan_partition_core(int32_t n_req, const int64_t *kv_lens, const int32_t *q_
     int32_t n_partials = 0;
     int32_t u = 0, tile = 0;  // next work: unit u from tile `tile` on; units that are in the pool are skipped
     while (u < U && units[u].pool_whole) ++u;
-    int64_t mean_overhead = 0;
-    for (int32_t i = 0; i < U; ++i) mean_overhead += units[i].overhead;
-    mean_overhead = U ? mean_overhead / U : 0;
     auto tiles_cost = [&](const Unit &un, int32_t from, int32_t to) -> int64_t {  // cost of tiles [from, to)
         if (to <= from) return 0;
         int64_t c = (int64_t)tune.tile_cost * (to - from);

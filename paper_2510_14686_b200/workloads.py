@@ -253,3 +253,36 @@ class PagedScenario:
             for r in finished:
                 a = admitted[r]
                 self.k[r], self.v[r], self.q_len[r] = a.k, a.v, a.q_len
+
+
+# --------------------------------------------------------------------------------------------
+# MLA (latent-attention) batches: per token one vector of d_c latent + d_r rotary dims shared by all
+# heads; per (query token, head) one query of the same width.  Values only, no arithmetic.
+# --------------------------------------------------------------------------------------------
+MLA_D_C = 512
+MLA_D_R = 64
+
+
+@dataclass
+class MlaBatch:
+    n_heads: int
+    q_lens: List[int]
+    kv_lens: List[int]
+    q: np.ndarray                                   # [sum q_len, n_heads, d_c + d_r] bf16 bit patterns
+    c: List[np.ndarray] = field(default_factory=list)  # per request [kv_len, d_c + d_r]
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / float(np.sqrt(128 + MLA_D_R))  # DeepSeek-style: softmax scale of the un-absorbed 128+64-dim heads
+
+
+def mla_batch(seed: int, n_heads: int, kv_lens: Sequence[int], q_lens: Optional[Sequence[int]] = None,
+              latent_std: float = 1.0, q_std: float = 0.25) -> MlaBatch:
+    """Seeded MLA batch.  Queries are drawn smaller than keys (absorbed queries are products of two projections;
+    with N(0,1) for both, 576-dim scores would make the softmax one-hot and hide mistakes in the weights)."""
+    q_lens = [1] * len(kv_lens) if q_lens is None else [int(x) for x in q_lens]
+    gen = torch.Generator().manual_seed(seed)
+    d = MLA_D_C + MLA_D_R
+    q = bf16_bits(torch.randn(sum(q_lens), n_heads, d, generator=gen, dtype=torch.float32) * q_std)
+    c = [bf16_bits(torch.randn(int(n), d, generator=gen, dtype=torch.float32) * latent_std) for n in kv_lens]
+    return MlaBatch(n_heads, q_lens, [int(n) for n in kv_lens], q, c)

@@ -51,6 +51,10 @@ typedef int32_t xllm_status;
 #define XLLM_FLAG_HOST_ONLY 4u         /* bookkeeping against an in-process fake of the driver: no GPU is touched, \
                                           every kernel-launching call returns XLLM_ERR_UNSUPPORTED (host tests) */
 
+#define XLLM_FLAG_MLA 8u               /* slots hold latent (MLA) caches: one 576-dim vector per token shared by all heads; \
+                                          needs n_kv_heads 1, head_dim 576, n_q_heads a multiple of 64; only the    \
+                                          xllm_mla_* calls compute on such a context, the mapper calls are unchanged */
+
 #define XLLM_TILE_TOKENS 64 /* tokens per KV tile block: unit of the private slot layout and of work splitting */
 #define XLLM_MAX_Q_LEN 8    /* upper bound accepted for xllm_config.max_q_len */
 
@@ -58,7 +62,7 @@ typedef struct {
     int32_t device;            /* CUDA device ordinal */
     int32_t n_q_heads;         /* H_q, a multiple of n_kv_heads */
     int32_t n_kv_heads;        /* H_kv */
-    int32_t head_dim;          /* D: 64 or 128 */
+    int32_t head_dim;          /* D: 64 or 128 (576 with XLLM_FLAG_MLA) */
     int32_t max_slots;         /* number of request slots (virtual ranges) */
     int32_t max_q_len;         /* largest q_len a verify call may carry, 1..XLLM_MAX_Q_LEN */
     int64_t max_seq_len;       /* tokens of virtual range per slot ("MaxSeqLen") */
@@ -333,6 +337,30 @@ xllm_status xllm_merge_partials(xllm_ctx *ctx, int32_t n_parts, int64_t n_rows, 
                                 void *out, float *lse_out, void *cuda_stream);
 
 /* ---- work partition (host only; exposed so that it can be checked without a GPU) ---------------------------- */
+
+/* ---- MLA: attention over latent caches ---------------------------------------------------------------------
+ * The report's own attention operator is multi-head latent attention rebuilt for contiguous virtual addresses
+ * ("Efficient Memory Management", Operator Adaptation), and speculative decoding gives it m+1 query tokens per
+ * sequence over the same K ("Algorithm Optimizations", MLA Optimization).  In the weight-absorbed decode form a
+ * token's cache entry is one bf16 vector c = [latent 512 | rotary key 64]; head h of a query token holds q of the
+ * same 576 dims; score = scale * <q, c>, value = the 512 latent dims.  Contexts created with XLLM_FLAG_MLA keep
+ * such vectors in their slots (1152 bytes per token); reserve / map / release / set_len work as for K/V caches.
+ *
+ * xllm_mla_append: c_new device bf16 [sum n_new, 576] (16-byte aligned), rows of request i follow those of i-1;
+ *   writes them at positions kv_len.. of each slot and advances kv_len.  Pages must be mapped (NOT_MAPPED else).
+ * xllm_mla_gather: copies tokens [first_token, first_token + n_tokens) of a slot back as dense [n_tokens, 576]
+ *   (the inverse of append; tests).
+ * xllm_mla_attention: q device bf16 [sum q_lens, H, 576], out device bf16 [sum q_lens, H, 512], lse_out device
+ *   fp32 [sum q_lens, H] (natural log) or NULL; q_lens NULL = one query token per request (decode), else the
+ *   newest q_len tokens of each slot are the query tokens (verification: token t sees kv_len - q_len + t + 1 keys).
+ *   Long sequences are split across CTAs and merged by their log-sum-exp weights.
+ * All three: asynchronous on cuda_stream, caller keeps the buffers alive until the stream has passed the call;
+ * errors as for the K/V calls (INVALID for bad arguments, UNSUPPORTED on a context without the flag). */
+xllm_status xllm_mla_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new, const void *c_new,
+                            void *cuda_stream);
+xllm_status xllm_mla_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int64_t n_tokens, void *c_out, void *cuda_stream);
+xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q, void *out,
+                               float *lse_out, float scale, void *cuda_stream);
 
 /* Split the step's KV tile blocks into per-CTA runs of near-equal cost (hierarchical DP load balance,
  * layer 3: equalise tokens per compute unit, split long sequences).  kv_lens / q_lens: host [n_req].

@@ -23,7 +23,8 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 OK, ERR_INVALID, ERR_OOM_PHYS, ERR_OOM_VA, ERR_NOT_MAPPED, ERR_CUDA, ERR_BUSY, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7
-FLAG_LAZY_PAGES, FLAG_NONBLOCKING_UNMAP, FLAG_HOST_ONLY = 1, 2, 4
+FLAG_LAZY_PAGES, FLAG_NONBLOCKING_UNMAP, FLAG_HOST_ONLY, FLAG_MLA = 1, 2, 4, 8
+MLA_LATENT, MLA_ROPE = 512, 64
 TILE_TOKENS = 64
 STATUS_NAMES = {0: "OK", -1: "INVALID", -2: "OOM_PHYS", -3: "OOM_VA", -4: "NOT_MAPPED", -5: "CUDA", -6: "BUSY",
                 -7: "UNSUPPORTED"}
@@ -107,6 +108,9 @@ EXPORTS = {
     "xllm_graph_step_destroy": (ctypes.c_int32, [_ctxp, ctypes.c_int32]),
     "xllm_partial_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_merge_partials": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, _vp, _vp, _vp, _vp, _vp]),
+    "xllm_mla_append": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp]),
+    "xllm_mla_gather": (ctypes.c_int32, [_ctxp, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, _vp, _vp]),
+    "xllm_mla_attention": (ctypes.c_int32, [_ctxp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp]),
     "xllm_plan_partition": (ctypes.c_int32, [ctypes.c_int32, _i64p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                               ctypes.POINTER(WorkItem), ctypes.c_int32, _i32p, _i32p, _i32p, _i32p]),
     "xllm_get_stats": (ctypes.c_int32, [_ctxp, ctypes.POINTER(Stats)]),
@@ -302,6 +306,20 @@ class Context:
         s, ql = _i32(slots), _i32(q_lens)
         self._check(_lib.xllm_verify_attention(self._ctx, len(s), s.ctypes.data, ql.ctypes.data, _ptr(q), _ptr(out),
                                                _ptr(lse_out), scale, _stream(stream)))
+
+    # -- MLA: latent caches (contexts created with FLAG_MLA) --
+    def mla_append(self, slots, n_new, c_new, stream=None):
+        s, n = _i32(slots), _i32(n_new)
+        self._check(_lib.xllm_mla_append(self._ctx, len(s), s.ctypes.data, n.ctypes.data, _ptr(c_new), _stream(stream)))
+
+    def mla_gather(self, slot: int, first_token: int, n_tokens: int, c_out, stream=None):
+        self._check(_lib.xllm_mla_gather(self._ctx, slot, first_token, n_tokens, _ptr(c_out), _stream(stream)))
+
+    def mla_attention(self, slots, q, out, lse_out=None, q_lens=None, scale: float = 1.0, stream=None):
+        s = _i32(slots)
+        ql = None if q_lens is None else _i32(q_lens)
+        self._check(_lib.xllm_mla_attention(self._ctx, len(s), s.ctypes.data, None if ql is None else ql.ctypes.data, _ptr(q),
+                                            _ptr(out), _ptr(lse_out), scale, _stream(stream)))
 
     # -- graph mode --
     def graph_step_create(self, q, out, lse_out=None, k_new=None, v_new=None, scale: float = 1.0) -> int:

@@ -9,8 +9,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libxllm_attn.so")
-SOURCES = ["api.cpp", "xtensor.cpp", "partition.cpp", "kernels.cu", "noalloc.cu"]
-HEADERS = ["xllm_internal.h", "xtensor.h", os.path.join(ROOT, "include", "xllm_attn.h")]
+SOURCES = ["api.cpp", "xtensor.cpp", "partition.cpp", "kernels.cu", "mla.cu", "noalloc.cu"]
+HEADERS = ["xllm_internal.h", "xtensor.h", "device_helpers.cuh", os.path.join(ROOT, "include", "xllm_attn.h")]
 
 
 def _stale() -> bool:

@@ -60,6 +60,9 @@ struct GraphStep {
 };
 
 struct xllm_ctx {
+    bool mla = false;  // XLLM_FLAG_MLA: slots hold one 576-dim latent vector per token; only the xllm_mla_* calls compute on them
+    std::vector<int64_t> mla_kv;      // per query token of an MLA call: keys it sees
+    std::vector<int32_t> mla_req;     // ... and the request it belongs to
     // One lock serialises every entry point and the pre-mapping worker (recursive: the fused append falls back to
     // xllm_kv_append from inside an attention call).
     std::recursive_mutex mu;
@@ -287,6 +290,7 @@ xllm_status attention_impl(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     XLLM_LOCK(ctx);
     const bool with_append = k_new != nullptr || v_new != nullptr;
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context is host-only, no GPU work possible");
+    if (ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context holds latent (MLA) caches; use the xllm_mla_* calls");
     xllm_status st = check_device_flag(ctx);
     if (st != XLLM_OK) return st;
     st = check_slot_list(ctx, n_req, slots, who);
@@ -505,7 +509,13 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     };
     if (cfg->n_kv_heads < 1 || cfg->n_q_heads < cfg->n_kv_heads || cfg->n_q_heads % cfg->n_kv_heads)
         return bad(XLLM_ERR_INVALID, "n_q_heads must be a positive multiple of n_kv_heads");
-    if (cfg->head_dim != 64 && cfg->head_dim != 128) return bad(XLLM_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    const bool mla = (cfg->flags & XLLM_FLAG_MLA) != 0;
+    if (mla) {
+        if (cfg->n_kv_heads != 1 || cfg->head_dim != kMlaDim || cfg->n_q_heads % kMlaRows)
+            return bad(XLLM_ERR_UNSUPPORTED, "XLLM_FLAG_MLA needs n_kv_heads 1, head_dim 576 (512 latent + 64 rotary) and n_q_heads a multiple of 64");
+    } else if (cfg->head_dim != 64 && cfg->head_dim != 128) {
+        return bad(XLLM_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+    }
     if (cfg->max_slots < 1 || cfg->max_seq_len < 1 || cfg->max_seq_len > (int64_t)INT32_MAX - XLLM_TILE_TOKENS)
         return bad(XLLM_ERR_INVALID, "max_slots and max_seq_len must be positive (max_seq_len < 2^31)");
     if (cfg->max_q_len < 1 || cfg->max_q_len > XLLM_MAX_Q_LEN) return bad(XLLM_ERR_INVALID, "max_q_len must be in [1, XLLM_MAX_Q_LEN]");
@@ -514,7 +524,8 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     std::unique_ptr<xllm_ctx> ctx(new xllm_ctx());
     ctx->cfg = *cfg;
     ctx->host_only = (cfg->flags & XLLM_FLAG_HOST_ONLY) != 0;
-    const int64_t row_bytes = 2ll * cfg->n_kv_heads * cfg->head_dim * 2;
+    ctx->mla = mla;
+    const int64_t row_bytes = mla ? (int64_t)kMlaDim * 2 : 2ll * cfg->n_kv_heads * cfg->head_dim * 2;
     std::unique_ptr<VmmDriver> drv;
     if (ctx->host_only) {
         drv = make_fake_driver(cfg->fault_inject);
@@ -556,7 +567,9 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     std::string perr;
     xllm_status st = ctx->xt->init_pool(cfg->phys_budget_bytes, cfg->page_bytes, (cfg->flags & XLLM_FLAG_LAZY_PAGES) != 0, &perr);
     if (st != XLLM_OK) return bad(st, perr);
-    if (ctx->xt->page_bytes() % ((int64_t)XLLM_TILE_TOKENS * row_bytes) != 0 &&
+    // (a latent tile block is 72 KiB and shares no factor structure with the page size: blocks may straddle pages, which
+    // the contiguous virtual range hides; tokens-to-pages arithmetic rounds up, capacity rounds down)
+    if (!mla && ctx->xt->page_bytes() % ((int64_t)XLLM_TILE_TOKENS * row_bytes) != 0 &&
         ((int64_t)XLLM_TILE_TOKENS * row_bytes) % ctx->xt->page_bytes() != 0)
         return bad(XLLM_ERR_UNSUPPORTED, "page size and tile block size must divide one another");
     xllm_ctx *raw = ctx.get();
@@ -578,8 +591,9 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
             if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&ctx->d_stage[i]), ctx->h_stage[i], 0);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->done[i], cudaEventDisableTiming);
         }
-        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * kMaxRows * cfg->head_dim);
-        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * kMaxRows);
+        const size_t part_rows = mla ? kMlaRows : kMaxRows, part_dim = mla ? kMlaLatent : cfg->head_dim;
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * part_rows * part_dim);
+        if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * part_rows);
         // arrival counters of split units, and one more word: the claim counter of the shared pool
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_counters), sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
         if (e == cudaSuccess) e = cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
@@ -593,7 +607,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
             e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_trace), tb);
             if (e == cudaSuccess) e = cudaMemset(ctx->d_trace, 0, tb);
         }
-        if (e == cudaSuccess) e = (cudaError_t)configure_kernels(cfg->head_dim);
+        if (e == cudaSuccess) e = (cudaError_t)(mla ? mla_configure_kernels() : configure_kernels(cfg->head_dim));
         if (e != cudaSuccess) {
             const std::string m = std::string("allocating the workspace: ") + cudaGetErrorString(e);
             xllm_shutdown(ctx.release());
@@ -829,6 +843,7 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
     if (!ctx) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "append: context is host-only, no GPU work possible");
+    if (ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "append: context holds latent (MLA) caches; use xllm_mla_append");
     xllm_status st = check_device_flag(ctx);
     if (st != XLLM_OK) return st;
     st = check_slot_list(ctx, n_req, slots, "append");
@@ -884,6 +899,7 @@ xllm_status xllm_kv_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int
     if (!ctx) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "gather: context is host-only, no GPU work possible");
+    if (ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "gather: context holds latent (MLA) caches; use xllm_mla_gather");
     if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "gather: slot is not live");
     if (!k_out || !v_out || (reinterpret_cast<uintptr_t>(k_out) & 15) || (reinterpret_cast<uintptr_t>(v_out) & 15))
         return fail(ctx, XLLM_ERR_INVALID, "gather: outputs must be non-null and 16-byte aligned");
@@ -933,6 +949,7 @@ xllm_status xllm_graph_step_create(xllm_ctx *ctx, const void *q, const void *k_n
     if (!ctx || !handle_out) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "graph_step_create: context is host-only, no GPU work possible");
+    if (ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "graph_step_create: not available for latent (MLA) caches");
     if (!q || !out || (k_new == nullptr) != (v_new == nullptr))
         return fail(ctx, XLLM_ERR_INVALID, "graph_step_create: q and out must be non-null; k_new and v_new both or neither");
     GraphStep *gs = new GraphStep();
@@ -1009,6 +1026,7 @@ xllm_status xllm_merge_partials(xllm_ctx *ctx, int32_t n_parts, int64_t n_rows, 
     if (!ctx) return XLLM_ERR_INVALID;
     XLLM_LOCK(ctx);
     if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "merge_partials: context is host-only, no GPU work possible");
+    if (ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "merge_partials: not available for latent (MLA) caches");
     const xllm_status st = check_device_flag(ctx);
     if (st != XLLM_OK) return st;
     if (n_parts < 1 || n_rows < 1 || !out_parts || !lse_parts || !out)
@@ -1020,6 +1038,192 @@ xllm_status xllm_merge_partials(xllm_ctx *ctx, int32_t n_parts, int64_t n_rows, 
                                      cuda_stream);
     if (e) return cuda_fail(ctx, "launching the merge kernel", e);
     ++ctx->st.kernel_launches;
+    return XLLM_OK;
+}
+
+// ---- MLA: latent caches --------------------------------------------------------------------------------------
+
+xllm_status xllm_mla_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *n_new, const void *c_new,
+                            void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "mla_append: context is host-only, no GPU work possible");
+    if (!ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "mla_append: context was not created with XLLM_FLAG_MLA");
+    xllm_status st = check_device_flag(ctx);
+    if (st != XLLM_OK) return st;
+    st = check_slot_list(ctx, n_req, slots, "mla_append");
+    if (st != XLLM_OK) return st;
+    if (!n_new || !c_new || (reinterpret_cast<uintptr_t>(c_new) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, "mla_append: n_new and c_new must be non-null, c_new 16-byte aligned");
+    int64_t rows = 0;
+    for (int32_t i = 0; i < n_req; ++i) {
+        if (n_new[i] < 0) return fail(ctx, XLLM_ERR_INVALID, "mla_append: negative n_new");
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        if (s.kv_len + n_new[i] > ctx->cfg.max_seq_len)
+            return fail(ctx, XLLM_ERR_INVALID, "mla_append: slot " + std::to_string(slots[i]) + " would exceed max_seq_len");
+        if (s.kv_len + n_new[i] > ctx->xt->mapped_tokens(slots[i]))
+            return fail(ctx, XLLM_ERR_NOT_MAPPED, "mla_append: slot " + std::to_string(slots[i]) + " has pages for " +
+                                                      std::to_string(ctx->xt->mapped_tokens(slots[i])) + " tokens, needs " +
+                                                      std::to_string(s.kv_len + n_new[i]) + "; call xllm_kv_map_pages first");
+        rows += n_new[i];
+    }
+    if (rows > INT32_MAX) return fail(ctx, XLLM_ERR_INVALID, "mla_append: too many rows");
+    if (rows == 0) return XLLM_OK;
+    int idx;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    AppendDesc *ad = reinterpret_cast<AppendDesc *>(ctx->h_stage[idx]);
+    int32_t row0 = 0, n_desc = 0, max_new = 0;
+    for (int32_t i = 0; i < n_req; ++i) {
+        max_new = std::max(max_new, n_new[i]);
+        if (n_new[i] == 0) continue;
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        ad[n_desc++] = {s.base, (int32_t)s.kv_len, row0, n_new[i], 0};
+        row0 += n_new[i];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    time_begin(ctx, 2, stream);
+    e = launch_mla_append(ad, n_desc, max_new, c_new, stream);
+    time_end(ctx, stream);
+    if (e) return cuda_fail(ctx, "launching the latent append kernel", e);
+    ctx->st.kernel_launches += (n_desc + kAppendBatch - 1) / kAppendBatch;
+    finish_launch(ctx, idx, stream);
+    for (int32_t i = 0; i < n_req; ++i) {
+        SlotRecord &s = ctx->xt->slot(slots[i]);
+        s.kv_len += n_new[i];
+        s.last_use = ctx->seq;
+    }
+    ctx->st.tokens_appended += rows;
+    return XLLM_OK;
+}
+
+xllm_status xllm_mla_gather(xllm_ctx *ctx, int32_t slot, int64_t first_token, int64_t n_tokens, void *c_out, void *cuda_stream) {
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, "mla_gather: context is host-only, no GPU work possible");
+    if (!ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, "mla_gather: context was not created with XLLM_FLAG_MLA");
+    if (!ctx->xt->valid_slot(slot) || !ctx->xt->slot(slot).live) return fail(ctx, XLLM_ERR_INVALID, "mla_gather: slot is not live");
+    if (!c_out || (reinterpret_cast<uintptr_t>(c_out) & 15)) return fail(ctx, XLLM_ERR_INVALID, "mla_gather: c_out must be non-null and 16-byte aligned");
+    SlotRecord &s = ctx->xt->slot(slot);
+    if (first_token < 0 || n_tokens < 0 || first_token + n_tokens > s.kv_len)
+        return fail(ctx, XLLM_ERR_INVALID, "mla_gather: token range outside [0, kv_len)");
+    if (n_tokens == 0) return XLLM_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int idx;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    e = launch_mla_gather(s.base, first_token, n_tokens, c_out, stream);
+    if (e) return cuda_fail(ctx, "launching the latent gather kernel", e);
+    ++ctx->st.kernel_launches;
+    finish_launch(ctx, idx, stream);
+    s.last_use = ctx->seq;
+    return XLLM_OK;
+}
+
+xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, const int32_t *q_lens, const void *q, void *out,
+                               float *lse_out, float scale, void *cuda_stream) {
+    const char *who = "mla_attention";
+    if (!ctx) return XLLM_ERR_INVALID;
+    XLLM_LOCK(ctx);
+    if (ctx->host_only) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context is host-only, no GPU work possible");
+    if (!ctx->mla) return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": context was not created with XLLM_FLAG_MLA");
+    xllm_status st = check_device_flag(ctx);
+    if (st != XLLM_OK) return st;
+    st = check_slot_list(ctx, n_req, slots, who);
+    if (st != XLLM_OK) return st;
+    if (!q || !out || (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+        return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q and out must be non-null and 16-byte aligned");
+    if (!(scale > 0.f) || !std::isfinite(scale)) return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": scale must be finite and > 0");
+
+    // One planner request per query token: token t of q_len sees kv_len - (q_len - 1 - t) keys.  The planner's "KV heads"
+    // are the blocks of 64 query heads, each with one row group (all of them read the same latent tiles).
+    std::vector<int64_t> &tok_kv = ctx->mla_kv;
+    std::vector<int32_t> &tok_req = ctx->mla_req;
+    tok_kv.clear();
+    tok_req.clear();
+    for (int32_t i = 0; i < n_req; ++i) {
+        const int32_t ql = q_lens ? q_lens[i] : 1;
+        const SlotRecord &s = ctx->xt->slot(slots[i]);
+        if (ql < 1 || ql > ctx->cfg.max_q_len)
+            return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": q_len of request " + std::to_string(i) + " outside [1, max_q_len]");
+        if (s.kv_len < ql)
+            return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": slot " + std::to_string(slots[i]) + " holds " + std::to_string(s.kv_len) +
+                                                   " tokens, fewer than q_len " + std::to_string(ql));
+        for (int32_t t = 0; t < ql; ++t) {
+            tok_kv.push_back(s.kv_len - (ql - 1 - t));
+            tok_req.push_back(i);
+        }
+    }
+    const int32_t n_tok = (int32_t)tok_kv.size();
+    const int32_t head_blocks = ctx->cfg.n_q_heads / kMlaRows;
+    int32_t n_units = 0, n_partials = 0;
+    PlanTuning tune = ctx->tune;
+    tune.pool_pct = 0;      // (no run-time pool in this kernel)
+    tune.row_overhead = 0;  // every item carries the same 64 rows
+    if (plan_partition(n_tok, tok_kv.data(), nullptr, head_blocks, head_blocks, ctx->sm_count, tune, ctx->items, ctx->cta_begin,
+                       &n_units, &n_partials, &ctx->plan_scratch) != 0)
+        return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
+    const int32_t n_items = (int32_t)ctx->items.size();
+    if (n_items > ctx->max_items || n_partials > ctx->max_partials)
+        return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": work list exceeds the workspace sized at init");
+    std::vector<CombineDesc> &combine = ctx->combine;
+    combine.clear();
+    for (const xllm_work_item &it : ctx->items)
+        if (it.partial_idx >= 0 && it.partial_idx == it.part_first)  // first piece of a split unit
+            combine.push_back({it.part_first, it.n_parts, it.req, it.kv_head * kMlaRows, 1, kMlaRows});
+
+    int idx = -1;
+    int e = acquire_stage(ctx, &idx);
+    if (e) return cuda_fail(ctx, "waiting for a staging buffer", e);
+    const size_t off_comb = align_up(sizeof(MlaItem) * (size_t)n_items, 16);
+    if (align_up(off_comb + sizeof(CombineDesc) * combine.size(), 16) > ctx->stage_bytes)
+        return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
+    char *h = ctx->h_stage[idx], *d = ctx->d_stage[idx];
+    MlaItem *mi = reinterpret_cast<MlaItem *>(h);
+    for (int32_t i = 0; i < n_items; ++i) {
+        const xllm_work_item &w = ctx->items[(size_t)i];
+        const SlotRecord &s = ctx->xt->slot(slots[tok_req[(size_t)w.req]]);
+        mi[i].kv = s.base;
+        mi[i].q_row = w.req;  // query tokens are packed in request order: the planner's request index is the row
+        mi[i].head0 = w.kv_head * kMlaRows;
+        mi[i].tile_begin = w.tile_begin;
+        mi[i].tile_end = w.tile_end;
+        mi[i].kv_end = (int32_t)tok_kv[(size_t)w.req];
+        mi[i].partial_idx = w.partial_idx;
+    }
+    if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    MlaLaunch ml{};
+    ml.items = reinterpret_cast<const MlaItem *>(d);
+    ml.q = q;
+    ml.out = out;
+    ml.lse_out = lse_out;
+    ml.part_o = ctx->d_part_o;
+    ml.part_lse = ctx->d_part_lse;
+    ml.error_flag = ctx->d_error;
+    ml.n_heads = ctx->cfg.n_q_heads;
+    ml.scale_log2 = scale * 1.4426950408889634f;
+    ml.n_ctas = ctx->sm_count;
+    std::memcpy(ml.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    time_begin(ctx, 0, stream);
+    e = launch_mla_attention(ml, stream);
+    time_end(ctx, stream);
+    if (e) return cuda_fail(ctx, "launching the latent attention kernel", e);
+    ++ctx->st.kernel_launches;
+    if (!combine.empty()) {
+        time_begin(ctx, 1, stream);
+        e = launch_mla_combine(reinterpret_cast<const CombineDesc *>(d + off_comb), (int32_t)combine.size(), ctx->d_part_o, ctx->d_part_lse,
+                               out, lse_out, ctx->cfg.n_q_heads, stream);
+        time_end(ctx, stream);
+        if (e) return cuda_fail(ctx, "launching the latent combine kernel", e);
+        ++ctx->st.kernel_launches;
+    }
+    finish_launch(ctx, idx, stream);
+    for (int32_t i = 0; i < n_req; ++i) ctx->xt->slot(slots[i]).last_use = ctx->seq;
+    ++ctx->st.attention_calls;
+    ctx->st.work_items += n_items;
+    ctx->st.partial_items += n_partials;
     return XLLM_OK;
 }
 

@@ -23,6 +23,7 @@
 #include <utility>
 
 #include "xllm_internal.h"
+#include "device_helpers.cuh"
 
 namespace xllm {
 namespace {
@@ -36,7 +37,6 @@ constexpr int kEpilogueThreads = kEpilogueWarps * 32;
 constexpr int kThreads = (kConsumerWarps + 1 + kEpilogueWarps) * 32;  // 384
 constexpr int kItemBatch = 64;
 constexpr int kPoolSlots = 4;   // records of the shared pool the producer may publish ahead of the other warps
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // a bounded wait gives up after 2 s
 
 template <int D>
 struct Cfg {
@@ -81,108 +81,6 @@ struct Cfg {
 // ---- PTX wrappers --------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// Hand-off of a buffer whose contents this thread has just loaded into registers: the arrival must not be issued before
-// the loads have delivered (a load still in flight would see what the other side writes next).  `after` is a value
-// computed from everything that was loaded; it is stored to a scratch word of shared memory first -- a real use, which
-// neither compiler nor assembler can drop, and which cannot issue before its operand exists -- and the arrival follows
-// in program order.  (An operand that only appears in a comment of the asm text is removed by the assembler.)
-__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, uint32_t after, uint32_t scratch) {
-    asm volatile("st.shared.b32 [%2], %1;\n\tmbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar), "r"(after), "r"(scratch) : "memory");
-}
-// The same without release semantics, for a thread that has global stores in flight (a releasing arrive may first wait
-// until those are performed).
-__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar, float after, uint32_t scratch) {
-    asm volatile("st.shared.f32 [%2], %1;\n\tmbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar), "f"(after), "r"(scratch)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up after kWaitLimitNs or as soon as another warp of the CTA gave up.  On failure the
-// CTA-wide abort flag (shared) and the host-visible error word are set and false is returned; callers then
-// skip their work but keep executing the barrier protocol so that no warp is left waiting.
-// (the waiting loop is kept out of line: the kernel has some twenty waits, most of them in its hottest loops, and the
-// instruction cache is a scarce resource here)
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
-    const unsigned long long t0 = globaltimer_ns();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            *reinterpret_cast<volatile int32_t *>(error_flag) = code;  // host-mapped word, read by the next API call
-            __threadfence_system();
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag,
-                                          int code) {
-    if (*abort_flag) return false;
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, error_flag, code);
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// 2^x by the hardware approximation (relative error about 2^-22, far below the bf16 rounding of what it feeds; inputs here
-// are <= 0 or -inf, results in [0, 1]): one instruction instead of the library routine's range handling, in the hottest loop.
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// Programmatic dependent launch: every kernel of the library is launched so that its blocks may become resident
-// while the previous kernel of the stream drains.  Nothing that kernel wrote (and nothing it may still read) is
-// touched before grid_dependency_wait(), which returns once the previous kernel has completed and flushed.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void group_bar(int group) {
     __syncwarp();  // the barrier instruction is warp-aligned: make sure the lanes have re-converged

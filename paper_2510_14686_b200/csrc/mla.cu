@@ -1,0 +1,408 @@
+// MLA (multi-head latent attention) decode / verification kernels of libxllm_attn.so (sm_100a), first version.
+//
+// The cache holds ONE vector per token, c = [latent (512 dims) | rotary key (64 dims)], shared by all heads; head h of
+// a query token carries q = [q_latent | q_rope] of the same 576 dims (weight-absorbed form).  Scores use all 576 dims,
+// values are the 512 latent dims.  A slot's range is a sequence of tile blocks of 64 tokens; a block is 9 panels of
+// [64 tokens][64 dims] bf16 (128 B per token row, 16-byte chunks XOR-swizzled by token & 7), 72 KiB, so that a tile
+// lands in shared memory with nine linear bulk copies and feeds ldmatrix without bank conflicts, as in the GQA kernel.
+//
+// One persistent CTA per SM walks its run of work items (64 heads of one query token x a range of tiles).  Warp 8
+// streams tiles into a two-stage ring (cp.async.bulk + mbarrier); warps 0-7 compute: warp (rb, ch) owns rows
+// 16 rb..16 rb+15; for Q.K^T it takes tokens 32 ch..32 ch+31 of the tile over all 576 dims (Q fragments come from
+// shared memory, they do not fit registers), the two halves agree on row maxima through shared memory and exchange
+// their bf16 weights, and for P.V the warp accumulates all 64 tokens into latent columns 256 ch..256 ch+255
+// (128 fp32 registers per thread).  The contraction runs on mma.sync m16n8k16: with 128 heads per token this path is
+// as much tensor- as HBM-bound, and a tcgen05/TMEM version of the two contractions is the step after this one.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <utility>
+
+#include "xllm_internal.h"
+#include "device_helpers.cuh"
+
+namespace xllm {
+namespace {
+
+constexpr int T = XLLM_TILE_TOKENS;                    // 64
+constexpr int kD = kMlaDim;                            // 576
+constexpr int kDv = kMlaLatent;                        // 512
+constexpr int kPanels = kD / 64;                       // 9
+constexpr int kTileBytes = kPanels * kPanelBytes;      // 73,728
+constexpr int kRows = kMlaRows;                        // 64 heads per item
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;        // + producer warp
+constexpr int kStages = 2;
+constexpr int kPPitch = T * 2 + 16;                    // bytes per row of the weight tile (padded against bank conflicts)
+
+constexpr int kOffQ = 0;                                         // 9 panels [64 rows][128 B], swizzled like a tile
+constexpr int kOffKV = kOffQ + kTileBytes;                       // [kStages] tiles
+constexpr int kOffP = kOffKV + kStages * kTileBytes;             // [64][kPPitch] bf16 weights of the current tile
+constexpr int kOffMx = kOffP + kRows * kPPitch;                  // [2][64] row maxima of the two token halves
+constexpr int kOffSum = kOffMx + 2 * kRows * 4;                  // [2][64] row sums of the two token halves
+constexpr int kOffBars = kOffSum + 2 * kRows * 4;                // full[kStages], empty[kStages]
+constexpr int kOffFlags = kOffBars + 2 * kStages * 8;            // [0] abort flag
+constexpr int kSmemBytes = kOffFlags + 16;
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+static_assert(kOffKV % 1024 == 0 && kOffP % 16 == 0, "alignment");
+
+__device__ __forceinline__ void consumer_bar() {
+    __syncwarp();
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid_constant__ MlaLaunch p) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
+    const uint32_t bar_full = smem_base + kOffBars, bar_empty = bar_full + kStages * 8;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + s * 8, 1);
+            mbar_init(bar_empty + s * 8, kConsumerWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    grid_launch_dependents();
+    grid_dependency_wait();  // the previous kernel of the stream may still write q or the slots
+
+    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
+    uint32_t fill = 0;  // tiles of this CTA so far: stage = fill % kStages, use = fill / kStages
+
+    if (warp == kConsumerWarps) {
+        // ================= producer =================
+        if (lane == 0) {
+            for (int i = item_lo; i < item_hi; ++i) {
+                const MlaItem it = p.items[i];
+                const char *kv = reinterpret_cast<const char *>(it.kv);
+                for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
+                    const uint32_t s = fill % kStages, ph = (fill / kStages) & 1;
+                    const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);   // 16-token steps that hold visible tokens
+                    if (!mbar_wait(bar_empty + s * 8, ph ^ 1, abort_flag, p.error_flag, 21)) continue;
+                    mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
+                    const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
+                    const char *src = kv + (int64_t)tile * kTileBytes;
+#pragma unroll
+                    for (int pn = 0; pn < kPanels; ++pn) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
+                }
+            }
+        }
+        return;
+    }
+
+    // ================= consumers =================
+    const int rb = warp & 3, ch = warp >> 2;
+    const int g8 = lane >> 2, q4 = lane & 3, swz = lane & 7;
+    float *mxs = reinterpret_cast<float *>(smem + kOffMx);
+    float *sums = reinterpret_cast<float *>(smem + kOffSum);
+    const uint32_t p_smem = smem_base + kOffP;
+    bool live = true;
+
+    for (int i = item_lo; i < item_hi; ++i) {
+        const MlaItem it = p.items[i];
+        consumer_bar();  // everybody is done with the previous item's query rows
+        {
+            // query rows of the item's 64 heads -> swizzled panels
+            const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.q) +
+                                                               ((int64_t)it.q_row * p.n_heads + it.head0) * (kD * 2));
+            constexpr int kChunks = kRows * (kD / 8);  // 4608 chunks of 16 bytes: 18 per thread
+#pragma unroll 6
+            for (int c = tid; c < kChunks; c += kConsumerThreads) {
+                const int r = c / (kD / 8), cc = c % (kD / 8);
+                const uint4 v = src[c];
+                *reinterpret_cast<uint4 *>(smem + kOffQ + (cc >> 3) * kPanelBytes + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = v;
+            }
+        }
+        consumer_bar();
+
+        float o[kDv / 2 / 8][4];  // 32 column blocks of 8: this warp's half of the latent dims
+#pragma unroll
+        for (int n = 0; n < kDv / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+        float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+
+        const uint32_t q_row_addr = smem_base + kOffQ + (rb * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * 128;
+        const int a_csel = lane >> 4;
+
+        for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
+            const uint32_t s_idx = fill % kStages, ph = (fill / kStages) & 1;
+            const uint32_t stage = smem_base + kOffKV + s_idx * kTileBytes;
+            const int tile_tok0 = tile * T;
+            const bool tail = tile_tok0 + T > it.kv_end;  // holds tokens past the visible end (stale or unfetched bytes)
+            live = __all_sync(0xffffffffu, mbar_wait(bar_full + s_idx * 8, ph, abort_flag, p.error_flag, 22)) && live;
+
+            // ---- scores of this warp's 16 rows x 32 tokens over 576 dims ----
+            float s[4][4];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+            if (live) {
+                const int kr = ch * 32 + (lane & 7) + ((lane >> 4) << 3);
+                const int k_csel = (lane >> 3) & 1;
+                const uint32_t k_row_addr = stage + kr * 128;
+#pragma unroll 4
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    uint32_t a[4], b0, b1, b2, b3, c0, c1, c2, c3;
+                    const int cga = 2 * ks + a_csel, cgk = 2 * ks + k_csel;
+                    ldsm_x4(a[0], a[1], a[2], a[3], q_row_addr + (cga >> 3) * kPanelBytes + (((cga & 7) ^ swz) << 4));
+                    const uint32_t koff = (cgk >> 3) * kPanelBytes + (((cgk & 7) ^ swz) << 4);
+                    ldsm_x4(b0, b1, b2, b3, k_row_addr + koff);
+                    ldsm_x4(c0, c1, c2, c3, k_row_addr + 16 * 128 + koff);
+                    mma_bf16(s[0], a, b0, b1);
+                    mma_bf16(s[1], a, b2, b3);
+                    mma_bf16(s[2], a, c0, c1);
+                    mma_bf16(s[3], a, c2, c3);
+                }
+                if (tail) {
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int tok = tile_tok0 + ch * 32 + nt * 8 + 2 * q4 + (e & 1);
+                            if (tok >= it.kv_end) s[nt][e] = -INFINITY;
+                        }
+                }
+                mx0 = fmaxf(fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])), fmaxf(fmaxf(s[2][0], s[2][1]), fmaxf(s[3][0], s[3][1])));
+                mx1 = fmaxf(fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3])), fmaxf(fmaxf(s[2][2], s[2][3]), fmaxf(s[3][2], s[3][3])));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            }
+            if (q4 == 0) {
+                mxs[ch * kRows + rb * 16 + g8] = mx0;
+                mxs[ch * kRows + rb * 16 + g8 + 8] = mx1;
+            }
+            consumer_bar();  // (1) both halves' row maxima are visible
+
+            // ---- running max, weights of this half, exchange of the bf16 weight tile ----
+            mx0 = fmaxf(mxs[rb * 16 + g8], mxs[kRows + rb * 16 + g8]);
+            mx1 = fmaxf(mxs[rb * 16 + g8 + 8], mxs[kRows + rb * 16 + g8 + 8]);
+            const float mn0 = fmaxf(m[0], mx0 * p.scale_log2), mn1 = fmaxf(m[1], mx1 * p.scale_log2);
+            const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+            const float a0 = fast_exp2(m[0] - ms0), a1 = fast_exp2(m[1] - ms1);
+            m[0] = mn0;
+            m[1] = mn1;
+            l[0] *= a0;
+            l[1] *= a1;
+            if (live) {
+                const uint32_t dst = p_smem + (rb * 16 + g8) * kPPitch + (ch * 32 + 2 * q4) * 2;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    const float p0 = fast_exp2(fmaf(s[nt][0], p.scale_log2, -ms0)), p1 = fast_exp2(fmaf(s[nt][1], p.scale_log2, -ms0));
+                    const float p2 = fast_exp2(fmaf(s[nt][2], p.scale_log2, -ms1)), p3 = fast_exp2(fmaf(s[nt][3], p.scale_log2, -ms1));
+                    l[0] += p0 + p1;
+                    l[1] += p2 + p3;
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + nt * 16), "r"(pack_bf16(p0, p1)) : "memory");
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + 8 * kPPitch + nt * 16), "r"(pack_bf16(p2, p3)) : "memory");
+                }
+            }
+            if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {  // the running maximum moved: rescale the accumulator
+#pragma unroll
+                for (int n = 0; n < kDv / 16; ++n) {
+                    o[n][0] *= a0;
+                    o[n][1] *= a0;
+                    o[n][2] *= a1;
+                    o[n][3] *= a1;
+                }
+            }
+            consumer_bar();  // (2) the weight tile is complete
+
+            // ---- O[16 rows, 256 latent columns] += P[16 x 64] . C[64 x 256] ----
+            if (live) {
+                const int n_ks = tail ? min(4, (it.kv_end - tile_tok0 + 15) >> 4) : 4;  // 16-token steps that were fetched
+                const uint32_t p_addr = p_smem + (rb * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * kPPitch + ((lane >> 4) << 4);
+                const int vr = (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int v_csel = lane >> 4;
+#pragma unroll 1
+                for (int kk = 0; kk < n_ks; ++kk) {
+                    uint32_t pa[4];
+                    ldsm_x4(pa[0], pa[1], pa[2], pa[3], p_addr + kk * 32);
+                    uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
+                    if (tail) {  // rows never written may hold anything: force them to zero (0 * NaN would poison O)
+                        const int t0 = tile_tok0 + kk * 16 + 2 * q4;
+                        vmask0 = (t0 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < it.kv_end ? 0xffff0000u : 0u);
+                        vmask1 = (t0 + 8 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < it.kv_end ? 0xffff0000u : 0u);
+                    }
+                    const uint32_t row_addr = stage + (kk * 16 + vr) * 128;
+#pragma unroll
+                    for (int n2 = 0; n2 < kDv / 32; ++n2) {
+                        const int cg = ch * (kDv / 16) + 2 * n2 + v_csel;  // 8-column chunk of the latent dims
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
+                        b0 &= vmask0;
+                        b1 &= vmask1;
+                        b2 &= vmask0;
+                        b3 &= vmask1;
+                        mma_bf16(o[2 * n2], pa, b0, b1);
+                        mma_bf16(o[2 * n2 + 1], pa, b2, b3);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + s_idx * 8);  // this warp is done with the stage
+        }
+
+        // ---- end of the item: row sums of the two halves, then the result ----
+        l[0] += __shfl_xor_sync(0xffffffffu, l[0], 1);
+        l[0] += __shfl_xor_sync(0xffffffffu, l[0], 2);
+        l[1] += __shfl_xor_sync(0xffffffffu, l[1], 1);
+        l[1] += __shfl_xor_sync(0xffffffffu, l[1], 2);
+        if (q4 == 0) {
+            sums[ch * kRows + rb * 16 + g8] = l[0];
+            sums[ch * kRows + rb * 16 + g8 + 8] = l[1];
+        }
+        consumer_bar();
+        const float lt0 = sums[rb * 16 + g8] + sums[kRows + rb * 16 + g8];
+        const float lt1 = sums[rb * 16 + g8 + 8] + sums[kRows + rb * 16 + g8 + 8];
+        const float inv0 = lt0 > 0.f ? 1.f / lt0 : 0.f, inv1 = lt1 > 0.f ? 1.f / lt1 : 0.f;
+        if (live) {
+            const int r0 = rb * 16 + g8, r1 = r0 + 8;
+            if (it.partial_idx < 0) {
+                __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.out);
+                const int64_t base0 = ((int64_t)it.q_row * p.n_heads + it.head0 + r0) * kDv + ch * (kDv / 2) + 2 * q4;
+                const int64_t base1 = base0 + 8ll * kDv;
+#pragma unroll
+                for (int n = 0; n < kDv / 16; ++n) {
+                    *reinterpret_cast<uint32_t *>(out + base0 + n * 8) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
+                    *reinterpret_cast<uint32_t *>(out + base1 + n * 8) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
+                }
+                if (p.lse_out && ch == 0 && q4 == 0) {  // natural log
+                    p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r0] = lt0 > 0.f ? m[0] * 0.6931471805599453f + logf(lt0) : -INFINITY;
+                    p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r1] = lt1 > 0.f ? m[1] * 0.6931471805599453f + logf(lt1) : -INFINITY;
+                }
+            } else {
+                float *po = p.part_o + (int64_t)it.partial_idx * kRows * kDv;
+                const int64_t base0 = (int64_t)r0 * kDv + ch * (kDv / 2) + 2 * q4, base1 = base0 + 8ll * kDv;
+#pragma unroll
+                for (int n = 0; n < kDv / 16; ++n) {
+                    *reinterpret_cast<float2 *>(po + base0 + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+                    *reinterpret_cast<float2 *>(po + base1 + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+                }
+                if (ch == 0 && q4 == 0) {  // log2 domain
+                    p.part_lse[(int64_t)it.partial_idx * kRows + r0] = lt0 > 0.f ? m[0] + log2f(lt0) : -INFINITY;
+                    p.part_lse[(int64_t)it.partial_idx * kRows + r1] = lt1 > 0.f ? m[1] + log2f(lt1) : -INFINITY;
+                }
+            }
+        }
+    }
+}
+
+// One block per (row of a split unit): merges the unit's partial results by their log-sum-exp weights.
+__global__ void __launch_bounds__(kDv / 4) mla_combine_kernel(const CombineDesc *__restrict__ descs, const float *__restrict__ part_o,
+                                                              const float *__restrict__ part_lse, __nv_bfloat16 *__restrict__ out,
+                                                              float *__restrict__ lse_out, int n_heads) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const CombineDesc d = descs[blockIdx.y];
+    const int r = blockIdx.x, c4 = threadIdx.x;
+    float M = -INFINITY;
+    for (int k = 0; k < d.n_parts; ++k) M = fmaxf(M, part_lse[(int64_t)(d.partial_begin + k) * kRows + r]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float W = 0.f;
+    for (int k = 0; k < d.n_parts; ++k) {
+        const float ls = part_lse[(int64_t)(d.partial_begin + k) * kRows + r];
+        const float w = (ls == -INFINITY) ? 0.f : exp2f(ls - M);
+        W += w;
+        if (w > 0.f) {
+            const float4 v = *reinterpret_cast<const float4 *>(part_o + ((int64_t)(d.partial_begin + k) * kRows + r) * kDv + c4 * 4);
+            acc.x += w * v.x;
+            acc.y += w * v.y;
+            acc.z += w * v.z;
+            acc.w += w * v.w;
+        }
+    }
+    const float inv = W > 0.f ? 1.f / W : 0.f;
+    const int64_t row = (int64_t)d.out_row0 * n_heads + d.head0 + r;
+    *reinterpret_cast<uint2 *>(out + row * kDv + c4 * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+    if (c4 == 0 && lse_out) lse_out[row] = W > 0.f ? M * 0.6931471805599453f + logf(W) : -INFINITY;
+}
+
+// ---- append ("write_kvcache") of latent rows and its inverse: one thread moves one 16-byte chunk ----
+__device__ __forceinline__ int64_t mla_chunk_offset(int64_t pos, int c) {
+    const int64_t blk = pos / T;
+    const int r = (int)(pos % T);
+    return blk * kTileBytes + (c >> 3) * kPanelBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+}
+
+__global__ void mla_append_kernel(const __grid_constant__ AppendLaunch descs, const uint4 *__restrict__ c_new) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const AppendDesc d = descs.d[blockIdx.y];
+    constexpr int cpr = kD / 8;  // 72 chunks per token
+    const int64_t total = (int64_t)d.n_new * cpr;
+    for (int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; id < total; id += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(id % cpr);
+        const int row = (int)(id / cpr);
+        *reinterpret_cast<uint4 *>(d.base + mla_chunk_offset((int64_t)d.pos0 + row, c)) = c_new[(int64_t)d.row0 * cpr + id];
+    }
+}
+
+__global__ void mla_gather_kernel(uint64_t base, int64_t first_token, int64_t n_tokens, uint4 *__restrict__ c_out) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    constexpr int cpr = kD / 8;
+    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= n_tokens * cpr) return;
+    c_out[id] = *reinterpret_cast<const uint4 *>(base + mla_chunk_offset(first_token + id / cpr, (int)(id % cpr)));
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+}  // namespace
+
+int mla_configure_kernels() {
+    return (int)cudaFuncSetAttribute(mla_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+int launch_mla_attention(const MlaLaunch &p, void *stream) {
+    return (int)launch_pdl(mla_attention_kernel, dim3(p.n_ctas), dim3(kThreads), kSmemBytes, static_cast<cudaStream_t>(stream), p);
+}
+
+int launch_mla_combine(const CombineDesc *descs, int32_t n_units, const float *part_o, const float *part_lse, void *out,
+                       float *lse_out, int32_t n_heads, void *stream) {
+    return (int)launch_pdl(mla_combine_kernel, dim3(kRows, (unsigned)n_units), dim3(kDv / 4), 0, static_cast<cudaStream_t>(stream), descs,
+                           part_o, part_lse, static_cast<__nv_bfloat16 *>(out), lse_out, (int)n_heads);
+}
+
+int launch_mla_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *c_new, void *stream) {
+    const int64_t per_req = (int64_t)max_new * (kD / 8);
+    const int threads = 256;
+    const int64_t bx = std::min<int64_t>((per_req + threads - 1) / threads, 4096);
+    for (int32_t first = 0; first < n_req; first += kAppendBatch) {
+        const int32_t n = std::min(kAppendBatch, n_req - first);
+        AppendLaunch al;
+        for (int32_t i = 0; i < n; ++i) al.d[i] = descs[first + i];
+        const cudaError_t e = launch_pdl(mla_append_kernel, dim3((unsigned)bx, (unsigned)n), dim3(threads), 0,
+                                         static_cast<cudaStream_t>(stream), al, static_cast<const uint4 *>(c_new));
+        if (e != cudaSuccess) return (int)e;
+    }
+    return 0;
+}
+
+int launch_mla_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *c_out, void *stream) {
+    const int64_t total = n_tokens * (kD / 8);
+    const int threads = 256;
+    return (int)launch_pdl(mla_gather_kernel, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0,
+                           static_cast<cudaStream_t>(stream), base, first_token, n_tokens, static_cast<uint4 *>(c_out));
+}
+
+}  // namespace xllm

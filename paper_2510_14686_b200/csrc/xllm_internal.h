@@ -157,6 +157,37 @@ struct CombineLaunch {
     int32_t out_f32;
 };
 
+// ---- MLA (latent attention) path: one 576-dim vector per token shared by all heads -------------------------
+constexpr int32_t kMlaLatent = 512;              // latent dims: scored and used as the value
+constexpr int32_t kMlaRope = 64;                 // rotary key dims: scored only
+constexpr int32_t kMlaDim = kMlaLatent + kMlaRope;
+constexpr int32_t kMlaRows = 64;                 // heads one work item carries (one query token)
+inline int64_t mla_tile_block_bytes() { return (int64_t)(kMlaDim / 64) * kPanelBytes; }  // 9 panels, 72 KiB per 64 tokens
+
+struct MlaItem {            // one work item: 64 heads of one query token over a range of tiles (32 bytes)
+    uint64_t kv;            // address of tile block 0 of the slot's range
+    int32_t q_row;          // the query token's row in q / out
+    int32_t head0;          // first of the item's 64 heads
+    int32_t tile_begin, tile_end;
+    int32_t kv_end;         // keys visible to the query token
+    int32_t partial_idx;    // -1: writes the final output; else slot in the partial workspace
+};
+static_assert(sizeof(MlaItem) == 32, "MlaItem layout");
+
+struct MlaLaunch {
+    const MlaItem *items;   // device-visible, grouped by CTA
+    const void *q;          // [rows, n_heads, 576] bf16
+    void *out;              // [rows, n_heads, 512] bf16
+    float *lse_out;         // [rows, n_heads] natural log, may be null
+    float *part_o;          // [n_partials][64][512] fp32, normalised
+    float *part_lse;        // [n_partials][64] (log2 domain)
+    int32_t *error_flag;    // host-mapped; set non-zero when a bounded wait expires
+    int32_t n_heads;
+    float scale_log2;
+    int32_t n_ctas;
+    int32_t cta_begin[kMaxCtas + 1];
+};
+
 constexpr int32_t kTraceWords = 16;  // per-CTA words of the optional trace buffer
 
 // kernels.cu
@@ -174,5 +205,13 @@ int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const
                   int32_t n_kv_heads, int32_t head_dim, void *stream);
 int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_out, void *v_out, int32_t n_kv_heads,
                   int32_t head_dim, void *stream);
+
+// mla.cu
+int mla_configure_kernels();
+int launch_mla_attention(const MlaLaunch &p, void *stream);
+int launch_mla_combine(const CombineDesc *descs, int32_t n_units, const float *part_o, const float *part_lse, void *out,
+                       float *lse_out, int32_t n_heads, void *stream);
+int launch_mla_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *c_new, void *stream);
+int launch_mla_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *c_out, void *stream);
 
 }  // namespace xllm

@@ -1,0 +1,178 @@
+"""GPU: MLA (latent-cache) append / gather byte checks and attention parity against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mla_oracle
+from paper_2510_14686_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+D = wl.MLA_D_C + wl.MLA_D_R
+PAGE = 2 << 20
+MAX_ABS, MEAN_ABS, LSE_ABS = 1e-2, 1e-3, 1e-3   # bf16 output vs fp64 oracle, latent values ~ N(0,1)
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_14686_b200 import binding as b
+
+    return b
+
+
+def mla_ctx(binding, n_heads, n_slots, max_seq_len, kv_lens, max_q_len=4):
+    pages = sum(-(-(-(-int(t) // 64) * 64 * D * 2) // PAGE) for t in kv_lens) + 2
+    return binding.Context(n_heads, 1, D, n_slots, max_seq_len, pages * PAGE, max_q_len=max_q_len, flags=binding.FLAG_MLA)
+
+
+def load(ctx, batch):
+    from gpu_harness import dev_bits
+
+    slots = []
+    for c in batch.c:
+        s = ctx.kv_reserve(expected_tokens=len(c))
+        ctx.kv_map_pages(s, len(c))
+        ctx.mla_append([s], [len(c)], dev_bits(c))
+        slots.append(s)
+    ctx.sync_check()
+    return slots
+
+
+def run(ctx, batch, slots, decode_call=False):
+    from gpu_harness import dev_bits, host_bits
+
+    q = dev_bits(batch.q)
+    rows = q.shape[0]
+    out = torch.zeros((rows, batch.n_heads, wl.MLA_D_C), dtype=torch.int16, device="cuda")
+    lse = torch.full((rows, batch.n_heads), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.mla_attention(slots, q, out, lse, None if decode_call else batch.q_lens, batch.scale)
+    ctx.sync_check()
+    return host_bits(out), lse.cpu().numpy()
+
+
+def check(batch, out_bits, lse):
+    ref_o, ref_l = mla_oracle.mla_attention_batch(batch.q, batch.c, batch.q_lens, batch.scale, wl.MLA_D_C)
+    got = wl.bits_to_f64(out_bits)
+    assert got.shape == ref_o.shape and np.isfinite(got).all()
+    err = np.abs(got - ref_o)
+    assert err.max() <= MAX_ABS, f"max-abs {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+    assert err.mean() <= MEAN_ABS, f"mean-abs {err.mean():.3e}"
+    e = np.abs(lse.astype(np.float64) - ref_l)
+    assert e.max() <= LSE_ABS, f"lse max-abs {e.max():.3e} at {np.unravel_index(e.argmax(), e.shape)}"
+
+
+def test_latent_append_then_gather_is_bit_exact_across_pages(binding):
+    from gpu_harness import dev_bits, host_bits
+
+    rng = np.random.default_rng(576)
+    per_page = PAGE // (D * 2)
+    total = 2 * per_page + 77                       # three pages; 72 KiB tile blocks straddle the page borders
+    c = rng.integers(0, 1 << 16, (total, D), dtype=np.uint16)
+    with binding.Context(128, 1, D, 2, total + 100, 8 * PAGE, flags=binding.FLAG_MLA) as ctx:
+        s = ctx.kv_reserve()
+        done = 0
+        for n in (1, 63, 64, per_page - 100, 300, total - per_page - 328):   # ragged appends, each after mapping its pages
+            ctx.kv_map_pages(s, done + n)
+            ctx.mla_append([s], [n], dev_bits(c[done:done + n]))
+            done += n
+        assert done == total and ctx.kv_slot_info(s).kv_len == total and ctx.kv_slot_info(s).row_bytes == D * 2
+        back = torch.zeros((total, D), dtype=torch.int16, device="cuda")
+        ctx.mla_gather(s, 0, total, back)
+        ctx.sync_check()
+        assert np.array_equal(host_bits(back), c)
+        part = torch.zeros((100, D), dtype=torch.int16, device="cuda")
+        ctx.mla_gather(s, per_page - 50, 100, part)  # a window across the first page border
+        ctx.sync_check()
+        assert np.array_equal(host_bits(part), c[per_page - 50:per_page + 50])
+
+
+@pytest.mark.parametrize("n_heads", [64, 128])
+def test_decode_parity_ragged_lengths(binding, n_heads):
+    kv = [1, 15, 63, 64, 65, 129, 200, 1000, 3001]     # single token, tile edges, several tiles with ragged tails
+    b = wl.mla_batch(2001 + n_heads, n_heads, kv)
+    with mla_ctx(binding, n_heads, len(kv), 4096, kv) as ctx:
+        slots = load(ctx, b)
+        out, lse = run(ctx, b, slots, decode_call=True)
+        check(b, out, lse)
+        out2, lse2 = run(ctx, b, slots)                # q_lens of ones: same plan, bitwise the same answer
+        assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_verification_parity_causal_tail(binding):
+    kv = [5, 64, 130, 700, 66, 4]
+    ql = [1, 3, 4, 2, 4, 4]                            # the last one: every query token's view ends inside the first tile
+    b = wl.mla_batch(2002, 128, kv, ql)
+    with mla_ctx(binding, 128, len(kv), 1024, kv) as ctx:
+        slots = load(ctx, b)
+        out, lse = run(ctx, b, slots)
+        check(b, out, lse)
+
+
+def test_long_sequences_are_split_and_merged(binding):
+    kv = [20000, 9000, 70]
+    ql = [1, 2, 1]
+    b = wl.mla_batch(2003, 128, kv, ql)
+    with mla_ctx(binding, 128, len(kv), 20480, kv) as ctx:
+        slots = load(ctx, b)
+        before = ctx.get_stats().as_dict()
+        out, lse = run(ctx, b, slots)
+        after = ctx.get_stats().as_dict()
+        assert after["partial_items"] > before["partial_items"]          # the split path really ran
+        assert after["kernel_launches"] - before["kernel_launches"] == 2  # attention + combine
+        check(b, out, lse)
+        out2, lse2 = run(ctx, b, slots)
+        assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_many_requests_more_items_than_ctas(binding):
+    rng = np.random.default_rng(2004)
+    kv = [int(x) for x in rng.integers(1, 400, 200)]
+    b = wl.mla_batch(2004, 128, kv)
+    with mla_ctx(binding, 128, len(kv), 512, kv) as ctx:
+        slots = load(ctx, b)
+        out, lse = run(ctx, b, slots)
+        check(b, out, lse)
+
+
+def test_stale_bytes_past_the_end_do_not_leak(binding):
+    from gpu_harness import dev_bits
+
+    # fill a slot with NaN patterns, shrink it, then write a shorter sequence: the kernel fetches whole 16-token steps
+    kv = [37]
+    b = wl.mla_batch(2005, 64, kv)
+    with mla_ctx(binding, 64, 1, 256, [128]) as ctx:
+        s = ctx.kv_reserve()
+        ctx.kv_map_pages(s, 128)
+        ctx.mla_append([s], [128], dev_bits(np.full((128, D), 0x7FC0, dtype=np.uint16)))   # bf16 NaN everywhere
+        ctx.kv_set_len(s, 0)
+        ctx.mla_append([s], [37], dev_bits(b.c[0]))
+        out, lse = run(ctx, b, [s])
+        check(b, out, lse)
+
+
+def test_modes_refuse_each_others_calls(binding):
+    from gpu_harness import dev_bits
+
+    z = torch.zeros((4, 128, D), dtype=torch.int16, device="cuda")
+    with binding.Context(128, 1, D, 1, 256, 4 * PAGE, flags=binding.FLAG_MLA) as ctx:
+        s = ctx.kv_reserve()
+        ctx.kv_map_pages(s, 4)
+        with pytest.raises(binding.XllmError) as e:
+            ctx.kv_append([s], [1], z, z)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        with pytest.raises(binding.XllmError) as e:
+            ctx.decode_attention([s], z, z)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        with pytest.raises(binding.XllmError) as e:    # no tokens yet
+            ctx.mla_attention([s], z, z)
+        assert e.value.status == binding.ERR_INVALID
+    with binding.Context(8, 2, 64, 1, 256, 4 * PAGE) as ctx:
+        s = ctx.kv_reserve()
+        with pytest.raises(binding.XllmError) as e:
+            ctx.mla_append([s], [1], z)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+        with pytest.raises(binding.XllmError) as e:
+            ctx.mla_attention([s], z, z)
+        assert e.value.status == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.XllmError):             # wrong geometry for the flag
+        binding.Context(100, 1, D, 1, 256, 4 * PAGE, flags=binding.FLAG_MLA)

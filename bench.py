@@ -385,6 +385,92 @@ def run_graph(args):
                       "hbm_gbs_whole_step": kv_bytes / (ms * 1e-3) / 1e9, "gpu_launches": 2 * args.steps}))
 
 
+def run_mla(args):
+    """`--mla NAME`: the MLA (latent-cache) attention on a named synthetic batch; 1 GPU.  A side measurement of the path's
+    next row, not the headline: 128 heads share every cache byte, so the kernel is bound by the tensor pipe as much as by
+    HBM, and both fractions are reported."""
+    import torch
+
+    from paper_2510_14686_b200 import binding
+
+    torch.cuda.set_device(0)
+    name = args.mla
+    kv, ql = wl.mla_lengths(name)
+    B, H, D, DC = len(kv), wl.MLA_HEADS, wl.MLA_D_C + wl.MLA_D_R, wl.MLA_D_C
+    row_bytes = D * 2
+    page = 2 << 20
+    per_copy = int(sum(-(-(-(-int(t) // 64) * 64 * row_bytes) // page) for t in kv))
+    copies = max(2, -(-2 * L2_BYTES // (int(kv.sum()) * row_bytes)))       # successive steps read different bytes
+    ctx = binding.Context(H, 1, D, B * copies, int(kv.max()) + 64, (per_copy * copies + 4) * page, max_q_len=int(ql.max()),
+                          flags=binding.FLAG_MLA)
+    gen = torch.Generator(device="cuda").manual_seed(binding.MLA_LATENT + B)
+    slots = []
+    for c in range(copies):
+        ss = np.zeros(B, np.int32)
+        for r in range(B):
+            sl = ctx.kv_reserve(expected_tokens=int(kv[r]))
+            ctx.kv_map_pages(sl, int(kv[r]))
+            for t0 in range(0, int(kv[r]), 1 << 15):
+                n = min(int(kv[r]) - t0, 1 << 15)
+                ctx.mla_append([sl], [n], torch.randn((n, D), generator=gen, device="cuda").to(torch.bfloat16))
+            ss[r] = sl
+        slots.append(ss)
+    rows = int(ql.sum())
+    q = (torch.randn((rows, H, D), generator=gen, device="cuda") * 0.25).to(torch.bfloat16)
+    out = torch.zeros((rows, H, DC), dtype=torch.bfloat16, device="cuda")
+    scale = 1.0 / float(np.sqrt(128 + wl.MLA_D_R))
+    stream = torch.cuda.current_stream().cuda_stream
+    q_lens = None if int(ql.max()) == 1 else ql
+
+    def step(i):
+        ctx.mla_attention(slots[i % copies], q, out, None, q_lens, scale, stream)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    ctx.sync_check()
+    ctx.set_profiling(True)
+    st0 = ctx.get_stats().as_dict()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ctx.sync_check()
+    st1 = ctx.get_stats().as_dict()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    n_attn = max(1, st1["attn_launches"] - st0["attn_launches"])
+    attn_ms = (st1["attn_kernel_ms"] - st0["attn_kernel_ms"]) / n_attn
+    comb_ms = (st1["combine_kernel_ms"] - st0["combine_kernel_ms"]) / n_attn
+    # algorithmic work of one launch: every visible (query token, key) pair is scored over 576 dims and weighted over 512
+    pairs = int(sum(int(q_) * int(k) - int(q_) * (int(q_) - 1) // 2 for k, q_ in zip(kv, ql)))
+    flops = 2.0 * H * (D + DC) * pairs
+    kv_bytes = int(kv.sum()) * row_bytes
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            pk = json.load(f)
+        tf_peak, hbm_peak, which = float(pk["bf16_tflops_sustained"]), float(pk["hbm_gbs"]), "measured (sustained cuBLAS bf16; copy)"
+    except Exception:
+        tf_peak, hbm_peak, which = 1400.0, FALLBACK_HBM_GBS, "fallback"
+    tf = flops / (attn_ms * 1e-3) / 1e12
+    print(json.dumps({"metric": METRIC, "value": int(kv.sum()) / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+                      "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"mla_{name}: {B} sequences x {int(ql.max())} query tokens, {H} heads, latent 512 + rotary 64, "
+                                             f"contexts {int(kv.min())}..{int(kv.max())} tokens", "kv_copies_rotated": copies,
+                                 "kv_bytes_per_step_per_gpu": kv_bytes, "l2": "inputs larger than L2 (rotating KV copies)"},
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": tf_peak, "unit": "TFLOP/s", "frac": tf / tf_peak,
+                                   "traffic": None, "peak_source": which, "kernel": "mla_attention_kernel (mma.sync m16n8k16)",
+                                   "kernel_ms": attn_ms, "combine_kernel_ms": comb_ms, "flops_per_launch": flops,
+                                   "hbm_achieved_gbs": kv_bytes / (attn_ms * 1e-3) / 1e9,
+                                   "hbm_frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / hbm_peak},
+                      "gpu_launches": int(st1["kernel_launches"] - st0["kernel_launches"]), "clocks": clocks}))
+
+
 def run_ours(args):
     import torch
 
@@ -537,12 +623,13 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=list(wl.SHAPES), default="decode")
     ap.add_argument("--graph", action="store_true", help="side measurement: the step captured once, re-planned and replayed (1 GPU)")
+    ap.add_argument("--mla", choices=list(wl.MLA_WORKLOADS), default=None, help="side measurement: MLA attention over latent caches (1 GPU)")
     ap.add_argument("--split", type=int, default=1, help="side measurement: every sequence held as this many parts (1 GPU)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     else:
-        run_graph(args) if args.graph else run_split(args) if args.split > 1 else run_ours(args)
+        run_mla(args) if args.mla else run_graph(args) if args.graph else run_split(args) if args.split > 1 else run_ours(args)
 
 
 if __name__ == "__main__":

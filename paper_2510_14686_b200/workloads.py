@@ -286,3 +286,20 @@ def mla_batch(seed: int, n_heads: int, kv_lens: Sequence[int], q_lens: Optional[
     q = bf16_bits(torch.randn(sum(q_lens), n_heads, d, generator=gen, dtype=torch.float32) * q_std)
     c = [bf16_bits(torch.randn(int(n), d, generator=gen, dtype=torch.float32) * latent_std) for n in kv_lens]
     return MlaBatch(n_heads, q_lens, [int(n) for n in kv_lens], q, c)
+
+
+# Named MLA workloads (DeepSeek-style geometry: 128 heads, 512 + 64 dims): lengths only, seeded.
+MLA_HEADS = 128
+MLA_WORKLOADS = {
+    # name: (seed, batch, q_len, low, high)  -- context lengths uniform in [low, high]
+    "decode": (3001, 128, 1, 1024, 4096),    # mid-decode batch of 2k/2k-style conversations
+    "verify": (3002, 64, 4, 1024, 4096),     # m + 1 = 4 query tokens per sequence (speculative verification)
+    "long": (3003, 4, 1, 32768, 32768),      # few 32k-token sequences: every unit is split across CTAs
+}
+
+
+def mla_lengths(name: str):
+    seed, batch, q_len, lo, hi = MLA_WORKLOADS[name]
+    rng = np.random.default_rng(seed)
+    kv = rng.integers(lo, hi + 1, batch).astype(np.int64)
+    return kv, np.full(batch, q_len, dtype=np.int32)

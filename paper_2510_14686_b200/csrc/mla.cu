@@ -6,8 +6,12 @@
 // [64 tokens][64 dims] bf16 (128 B per token row, 16-byte chunks XOR-swizzled by token & 7), 72 KiB, so that a tile
 // lands in shared memory with nine linear bulk copies and feeds ldmatrix without bank conflicts, as in the GQA kernel.
 //
-// One persistent CTA per SM walks its run of work items (64 heads of one query token x a range of tiles).  Warp 8
-// streams tiles into a two-stage ring (cp.async.bulk + mbarrier); warps 0-7 compute: warp (rb, ch) owns rows
+// One persistent CTA per SM (8 warps, 255 registers per thread) walks its run of work items (64 heads of one query
+// token x a range of tiles).  Tiles arrive in a two-stage ring (cp.async.bulk + mbarrier transaction counts); one
+// elected thread issues the copy of tile f+1 right after the CTA-wide barrier in the middle of tile f, which every
+// warp reaches only when it is done with tile f-1, so the stage is free without a second set of barriers.  (A ninth,
+// copy-only warp would cap the kernel at 168 registers per thread: the register file is allocated as if the CTA had
+// 384 threads.)  Warp (rb, ch) owns rows
 // 16 rb..16 rb+15; for Q.K^T it takes tokens 32 ch..32 ch+31 of the tile over all 576 dims (Q fragments come from
 // shared memory, they do not fit registers), the two halves agree on row maxima through shared memory and exchange
 // their bf16 weights, and for P.V the warp accumulates all 64 tokens into latent columns 256 ch..256 ch+255
@@ -34,7 +38,7 @@ constexpr int kTileBytes = kPanels * kPanelBytes;      // 73,728
 constexpr int kRows = kMlaRows;                        // 64 heads per item
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;        // + producer warp
+constexpr int kThreads = kConsumerThreads;             // every warp computes; thread 0 also issues the copies
 constexpr int kStages = 2;
 constexpr int kPPitch = T * 2 + 16;                    // bytes per row of the weight tile (padded against bank conflicts)
 
@@ -43,58 +47,65 @@ constexpr int kOffKV = kOffQ + kTileBytes;                       // [kStages] ti
 constexpr int kOffP = kOffKV + kStages * kTileBytes;             // [64][kPPitch] bf16 weights of the current tile
 constexpr int kOffMx = kOffP + kRows * kPPitch;                  // [2][64] row maxima of the two token halves
 constexpr int kOffSum = kOffMx + 2 * kRows * 4;                  // [2][64] row sums of the two token halves
-constexpr int kOffBars = kOffSum + 2 * kRows * 4;                // full[kStages], empty[kStages]
-constexpr int kOffFlags = kOffBars + 2 * kStages * 8;            // [0] abort flag
-constexpr int kSmemBytes = kOffFlags + 16;
+constexpr int kOffBars = kOffSum + 2 * kRows * 4;                // full[kStages]
+constexpr int kOffFlags = kOffBars + kStages * 8;                // [0] abort flag
+constexpr int kItemCache = 16;                                   // item records kept in shared memory (the rest is read in place)
+constexpr int kOffItems = kOffFlags + 16;
+constexpr int kSmemBytes = kOffItems + kItemCache * (int)sizeof(MlaItem);
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 static_assert(kOffKV % 1024 == 0 && kOffP % 16 == 0, "alignment");
 
-__device__ __forceinline__ void consumer_bar() {
-    __syncwarp();
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-}
+__device__ __forceinline__ void consumer_bar() { __syncthreads(); }
 
 __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid_constant__ MlaLaunch p) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
-    const uint32_t bar_full = smem_base + kOffBars, bar_empty = bar_full + kStages * 8;
+    const uint32_t bar_full = smem_base + kOffBars;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full + s * 8, 1);
-            mbar_init(bar_empty + s * 8, kConsumerWarps);
-        }
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_full + s * 8, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
+    // The records live in host memory mapped into the device (a trip over PCIe each): the first ones are fetched once.
+    const MlaItem *sitems = reinterpret_cast<const MlaItem *>(smem + kOffItems);
+    if (tid < 2 * min(item_hi - item_lo, kItemCache))
+        reinterpret_cast<uint4 *>(smem + kOffItems)[tid] = reinterpret_cast<const uint4 *>(p.items + item_lo)[tid];
     __syncthreads();
     grid_launch_dependents();
     grid_dependency_wait();  // the previous kernel of the stream may still write q or the slots
+    auto item_at = [&](int i) -> MlaItem { return (i - item_lo < kItemCache) ? sitems[i - item_lo] : p.items[i]; };
 
-    const int item_lo = p.cta_begin[blockIdx.x], item_hi = p.cta_begin[blockIdx.x + 1];
     uint32_t fill = 0;  // tiles of this CTA so far: stage = fill % kStages, use = fill / kStages
 
-    if (warp == kConsumerWarps) {
-        // ================= producer =================
-        if (lane == 0) {
-            for (int i = item_lo; i < item_hi; ++i) {
-                const MlaItem it = p.items[i];
-                const char *kv = reinterpret_cast<const char *>(it.kv);
-                for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
-                    const uint32_t s = fill % kStages, ph = (fill / kStages) & 1;
-                    const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);   // 16-token steps that hold visible tokens
-                    if (!mbar_wait(bar_empty + s * 8, ph ^ 1, abort_flag, p.error_flag, 21)) continue;
-                    mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
-                    const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
-                    const char *src = kv + (int64_t)tile * kTileBytes;
+    // ---- copies (thread 0): a cursor over the CTA's tiles in order, one tile ahead of the computation ----
+    int c_item = item_lo, c_tile = 0;
+    uint32_t c_fill = 0;
+    MlaItem c_it = {};
+    if (tid == 0 && item_lo < item_hi) {
+        c_it = item_at(item_lo);
+        c_tile = c_it.tile_begin;
+    }
+    auto issue_next_tile = [&]() {  // thread 0 only; the stage it writes must be free
+        if (c_item >= item_hi) return;
+        const uint32_t s = c_fill % kStages;
+        const int rows = min(T, (c_it.kv_end - c_tile * T + 15) & ~15);  // 16-token steps that hold visible tokens
+        mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
+        const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
+        const char *src = reinterpret_cast<const char *>(c_it.kv) + (int64_t)c_tile * kTileBytes;
 #pragma unroll
-                    for (int pn = 0; pn < kPanels; ++pn) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
-                }
+        for (int pn = 0; pn < kPanels; ++pn) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
+        ++c_fill;
+        if (++c_tile >= c_it.tile_end) {
+            if (++c_item < item_hi) {
+                c_it = item_at(c_item);
+                c_tile = c_it.tile_begin;
             }
         }
-        return;
-    }
+    };
+    if (tid == 0) issue_next_tile();
 
     // ================= consumers =================
     const int rb = warp & 3, ch = warp >> 2;
@@ -105,7 +116,7 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
     bool live = true;
 
     for (int i = item_lo; i < item_hi; ++i) {
-        const MlaItem it = p.items[i];
+        const MlaItem it = item_at(i);
         consumer_bar();  // everybody is done with the previous item's query rows
         {
             // query rows of the item's 64 heads -> swizzled panels
@@ -145,18 +156,24 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                 const int kr = ch * 32 + (lane & 7) + ((lane >> 4) << 3);
                 const int k_csel = (lane >> 3) & 1;
                 const uint32_t k_row_addr = stage + kr * 128;
-#pragma unroll 4
-                for (int ks = 0; ks < kD / 16; ++ks) {
-                    uint32_t a[4], b0, b1, b2, b3, c0, c1, c2, c3;
+                // fragments of step ks+1 are fetched while the four MMAs of step ks run (fully unrolled: indices are constants)
+                uint32_t af[2][4], kf[2][8];
+                auto fetch = [&](int ks, int buf) {
                     const int cga = 2 * ks + a_csel, cgk = 2 * ks + k_csel;
-                    ldsm_x4(a[0], a[1], a[2], a[3], q_row_addr + (cga >> 3) * kPanelBytes + (((cga & 7) ^ swz) << 4));
+                    ldsm_x4(af[buf][0], af[buf][1], af[buf][2], af[buf][3], q_row_addr + (cga >> 3) * kPanelBytes + (((cga & 7) ^ swz) << 4));
                     const uint32_t koff = (cgk >> 3) * kPanelBytes + (((cgk & 7) ^ swz) << 4);
-                    ldsm_x4(b0, b1, b2, b3, k_row_addr + koff);
-                    ldsm_x4(c0, c1, c2, c3, k_row_addr + 16 * 128 + koff);
-                    mma_bf16(s[0], a, b0, b1);
-                    mma_bf16(s[1], a, b2, b3);
-                    mma_bf16(s[2], a, c0, c1);
-                    mma_bf16(s[3], a, c2, c3);
+                    ldsm_x4(kf[buf][0], kf[buf][1], kf[buf][2], kf[buf][3], k_row_addr + koff);
+                    ldsm_x4(kf[buf][4], kf[buf][5], kf[buf][6], kf[buf][7], k_row_addr + 16 * 128 + koff);
+                };
+                fetch(0, 0);
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    const int cur = ks & 1;
+                    if (ks + 1 < kD / 16) fetch(ks + 1, cur ^ 1);
+                    mma_bf16(s[0], af[cur], kf[cur][0], kf[cur][1]);
+                    mma_bf16(s[1], af[cur], kf[cur][2], kf[cur][3]);
+                    mma_bf16(s[2], af[cur], kf[cur][4], kf[cur][5]);
+                    mma_bf16(s[3], af[cur], kf[cur][6], kf[cur][7]);
                 }
                 if (tail) {
 #pragma unroll
@@ -178,7 +195,8 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                 mxs[ch * kRows + rb * 16 + g8] = mx0;
                 mxs[ch * kRows + rb * 16 + g8 + 8] = mx1;
             }
-            consumer_bar();  // (1) both halves' row maxima are visible
+            consumer_bar();  // (1) both halves' row maxima are visible; every warp is done with the tile before this one
+            if (tid == 0) issue_next_tile();  // ... so its stage takes the tile after this one
 
             // ---- running max, weights of this half, exchange of the bf16 weight tile ----
             mx0 = fmaxf(mxs[rb * 16 + g8], mxs[kRows + rb * 16 + g8]);
@@ -219,8 +237,9 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                 const uint32_t p_addr = p_smem + (rb * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * kPPitch + ((lane >> 4) << 4);
                 const int vr = (lane & 7) + (((lane >> 3) & 1) << 3);
                 const int v_csel = lane >> 4;
-#pragma unroll 1
-                for (int kk = 0; kk < n_ks; ++kk) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (kk >= n_ks) break;
                     uint32_t pa[4];
                     ldsm_x4(pa[0], pa[1], pa[2], pa[3], p_addr + kk * 32);
                     uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
@@ -244,8 +263,6 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty + s_idx * 8);  // this warp is done with the stage
         }
 
         // ---- end of the item: row sums of the two halves, then the result ----
@@ -291,6 +308,16 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
             }
         }
     }
+    // A wait ran out: before the CTA gives up its shared memory, give the copies still in flight a bounded time to land.
+    if (*abort_flag && tid == 0) {
+        for (uint32_t st = 0; st < kStages; ++st) {
+            const uint32_t uses = (c_fill + kStages - 1 - st) / kStages;  // copies issued into this stage so far
+            if (uses == 0) continue;
+            for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar_full + st * 8, (uses - 1) & 1); ++spin) {
+            }
+        }
+    }
+    __syncthreads();
 }
 
 // One block per (row of a split unit): merges the unit's partial results by their log-sum-exp weights.

@@ -95,6 +95,7 @@ struct xllm_ctx {
     cudaStream_t last_stream = nullptr;
 
     float *d_part_o = nullptr, *d_part_lse = nullptr;
+    CombineDesc *d_mla_comb = nullptr;  // MLA: device copy of a call's combine descriptors (written by its attention kernel)
     int32_t *d_counters = nullptr;  // arrival counters of split units (zero between launches)
     unsigned long long *d_trace = nullptr;  // per-CTA cycle counters, only when XLLM_TRACE is set in the environment
     int32_t max_partials = 0, max_items = 0;
@@ -593,6 +594,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
         }
         const size_t part_rows = mla ? kMlaRows : kMaxRows, part_dim = mla ? kMlaLatent : cfg->head_dim;
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_o), sizeof(float) * (size_t)ctx->max_partials * part_rows * part_dim);
+        if (e == cudaSuccess && mla) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_mla_comb), sizeof(CombineDesc) * (size_t)ctx->max_partials);
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_part_lse), sizeof(float) * (size_t)ctx->max_partials * part_rows);
         // arrival counters of split units, and one more word: the claim counter of the shared pool
         if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_counters), sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
@@ -634,6 +636,7 @@ xllm_status xllm_shutdown(xllm_ctx *ctx) {
             if (ctx->done[i]) cudaEventDestroy(ctx->done[i]);
         }
         if (ctx->d_part_o) cudaFree(ctx->d_part_o);
+        if (ctx->d_mla_comb) cudaFree(ctx->d_mla_comb);
         if (ctx->d_part_lse) cudaFree(ctx->d_part_lse);
         if (ctx->d_counters) cudaFree(ctx->d_counters);
         if (ctx->d_trace) cudaFree(ctx->d_trace);
@@ -1202,6 +1205,9 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ml.part_o = ctx->d_part_o;
     ml.part_lse = ctx->d_part_lse;
     ml.error_flag = ctx->d_error;
+    ml.comb_src = reinterpret_cast<const CombineDesc *>(d + off_comb);
+    ml.comb_dst = ctx->d_mla_comb;
+    ml.n_comb = (int32_t)combine.size();
     ml.n_heads = ctx->cfg.n_q_heads;
     ml.scale_log2 = scale * 1.4426950408889634f;
     ml.n_ctas = ctx->sm_count;
@@ -1213,7 +1219,7 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ++ctx->st.kernel_launches;
     if (!combine.empty()) {
         time_begin(ctx, 1, stream);
-        e = launch_mla_combine(reinterpret_cast<const CombineDesc *>(d + off_comb), (int32_t)combine.size(), ctx->d_part_o, ctx->d_part_lse,
+        e = launch_mla_combine(ctx->d_mla_comb, (int32_t)combine.size(), ctx->d_part_o, ctx->d_part_lse,
                                out, lse_out, ctx->cfg.n_q_heads, stream);
         time_end(ctx, stream);
         if (e) return cuda_fail(ctx, "launching the latent combine kernel", e);

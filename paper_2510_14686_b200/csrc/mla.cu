@@ -77,6 +77,9 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
     grid_launch_dependents();
     grid_dependency_wait();  // the previous kernel of the stream may still write q or the slots
     auto item_at = [&](int i) -> MlaItem { return (i - item_lo < kItemCache) ? sitems[i - item_lo] : p.items[i]; };
+    // The combine kernel that follows reads its descriptors many times: bring them from mapped host memory into device memory once.
+    for (int i = blockIdx.x * kThreads + tid; i < p.n_comb * (int)(sizeof(CombineDesc) / 8); i += p.n_ctas * kThreads)
+        reinterpret_cast<uint2 *>(p.comb_dst)[i] = reinterpret_cast<const uint2 *>(p.comb_src)[i];
 
     uint32_t fill = 0;  // tiles of this CTA so far: stage = fill % kStages, use = fill / kStages
 
@@ -320,34 +323,41 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
     __syncthreads();
 }
 
-// One block per (row of a split unit): merges the unit's partial results by their log-sum-exp weights.
-__global__ void __launch_bounds__(kDv / 4) mla_combine_kernel(const CombineDesc *__restrict__ descs, const float *__restrict__ part_o,
-                                                              const float *__restrict__ part_lse, __nv_bfloat16 *__restrict__ out,
-                                                              float *__restrict__ lse_out, int n_heads) {
+// Merge of split units by their log-sum-exp weights: block (u, y) handles rows 4y..4y+3 of unit u; a thread owns four
+// latent columns of one row at a time.
+constexpr int kCombineThreads = 256, kCombineRows = 4;
+__global__ void __launch_bounds__(kCombineThreads) mla_combine_kernel(const CombineDesc *__restrict__ descs, const float *__restrict__ part_o,
+                                                                      const float *__restrict__ part_lse, __nv_bfloat16 *__restrict__ out,
+                                                                      float *__restrict__ lse_out, int n_heads) {
     grid_launch_dependents();
     grid_dependency_wait();
-    const CombineDesc d = descs[blockIdx.y];
-    const int r = blockIdx.x, c4 = threadIdx.x;
-    float M = -INFINITY;
-    for (int k = 0; k < d.n_parts; ++k) M = fmaxf(M, part_lse[(int64_t)(d.partial_begin + k) * kRows + r]);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float W = 0.f;
-    for (int k = 0; k < d.n_parts; ++k) {
-        const float ls = part_lse[(int64_t)(d.partial_begin + k) * kRows + r];
-        const float w = (ls == -INFINITY) ? 0.f : exp2f(ls - M);
-        W += w;
-        if (w > 0.f) {
-            const float4 v = *reinterpret_cast<const float4 *>(part_o + ((int64_t)(d.partial_begin + k) * kRows + r) * kDv + c4 * 4);
-            acc.x += w * v.x;
-            acc.y += w * v.y;
-            acc.z += w * v.z;
-            acc.w += w * v.w;
+    const CombineDesc d = descs[blockIdx.x];
+    const int c4 = threadIdx.x & (kDv / 4 - 1);
+#pragma unroll
+    for (int rr = threadIdx.x / (kDv / 4); rr < kCombineRows; rr += kCombineThreads / (kDv / 4)) {
+        const int r = blockIdx.y * kCombineRows + rr;
+        float M = -INFINITY;
+        for (int k = 0; k < d.n_parts; ++k) M = fmaxf(M, part_lse[(int64_t)(d.partial_begin + k) * kRows + r]);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float W = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < d.n_parts; ++k) {
+            const float ls = part_lse[(int64_t)(d.partial_begin + k) * kRows + r];
+            const float w = (ls == -INFINITY) ? 0.f : exp2f(ls - M);
+            W += w;
+            if (w > 0.f) {
+                const float4 v = *reinterpret_cast<const float4 *>(part_o + ((int64_t)(d.partial_begin + k) * kRows + r) * kDv + c4 * 4);
+                acc.x += w * v.x;
+                acc.y += w * v.y;
+                acc.z += w * v.z;
+                acc.w += w * v.w;
+            }
         }
+        const float inv = W > 0.f ? 1.f / W : 0.f;
+        const int64_t row = (int64_t)d.out_row0 * n_heads + d.head0 + r;
+        *reinterpret_cast<uint2 *>(out + row * kDv + c4 * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        if (c4 == 0 && lse_out) lse_out[row] = W > 0.f ? M * 0.6931471805599453f + logf(W) : -INFINITY;
     }
-    const float inv = W > 0.f ? 1.f / W : 0.f;
-    const int64_t row = (int64_t)d.out_row0 * n_heads + d.head0 + r;
-    *reinterpret_cast<uint2 *>(out + row * kDv + c4 * 4) = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-    if (c4 == 0 && lse_out) lse_out[row] = W > 0.f ? M * 0.6931471805599453f + logf(W) : -INFINITY;
 }
 
 // ---- append ("write_kvcache") of latent rows and its inverse: one thread moves one 16-byte chunk ----
@@ -406,7 +416,7 @@ int launch_mla_attention(const MlaLaunch &p, void *stream) {
 
 int launch_mla_combine(const CombineDesc *descs, int32_t n_units, const float *part_o, const float *part_lse, void *out,
                        float *lse_out, int32_t n_heads, void *stream) {
-    return (int)launch_pdl(mla_combine_kernel, dim3(kRows, (unsigned)n_units), dim3(kDv / 4), 0, static_cast<cudaStream_t>(stream), descs,
+    return (int)launch_pdl(mla_combine_kernel, dim3((unsigned)n_units, kRows / kCombineRows), dim3(kCombineThreads), 0, static_cast<cudaStream_t>(stream), descs,
                            part_o, part_lse, static_cast<__nv_bfloat16 *>(out), lse_out, (int)n_heads);
 }
 

@@ -182,6 +182,9 @@ struct MlaLaunch {
     float *part_o;          // [n_partials][64][512] fp32, normalised
     float *part_lse;        // [n_partials][64] (log2 domain)
     int32_t *error_flag;    // host-mapped; set non-zero when a bounded wait expires
+    const CombineDesc *comb_src;  // descriptors of the split units in mapped host memory ...
+    CombineDesc *comb_dst;        // ... which the kernel copies here (device memory) for the combine kernel that follows
+    int32_t n_comb;
     int32_t n_heads;
     float scale_log2;
     int32_t n_ctas;

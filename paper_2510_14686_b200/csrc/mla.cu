@@ -47,8 +47,8 @@ constexpr int kOffKV = kOffQ + kTileBytes;                       // [kStages] ti
 constexpr int kOffP = kOffKV + kStages * kTileBytes;             // [64][kPPitch] bf16 weights of the current tile
 constexpr int kOffMx = kOffP + kRows * kPPitch;                  // [2][64] row maxima of the two token halves
 constexpr int kOffSum = kOffMx + 2 * kRows * 4;                  // [2][64] row sums of the two token halves
-constexpr int kOffBars = kOffSum + 2 * kRows * 4;                // full[kStages]
-constexpr int kOffFlags = kOffBars + kStages * 8;                // [0] abort flag
+constexpr int kOffBars = kOffSum + 2 * kRows * 4;                // full[kStages], empty[kStages]
+constexpr int kOffFlags = kOffBars + 2 * kStages * 8;            // [0] abort flag
 constexpr int kItemCache = 16;                                   // item records kept in shared memory (the rest is read in place)
 constexpr int kOffItems = kOffFlags + 16;
 constexpr int kSmemBytes = kOffItems + kItemCache * (int)sizeof(MlaItem);
@@ -56,15 +56,23 @@ static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA m
 static_assert(kOffKV % 1024 == 0 && kOffP % 16 == 0, "alignment");
 
 __device__ __forceinline__ void consumer_bar() { __syncthreads(); }
+// the two warps that share a block of 16 rows (token halves in Q.K^T, latent-column halves in P.V)
+__device__ __forceinline__ void pair_bar(int rb) {
+    __syncwarp();
+    asm volatile("bar.sync %0, 64;" ::"r"(rb + 1) : "memory");
+}
 
 __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid_constant__ MlaLaunch p) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffFlags);
-    const uint32_t bar_full = smem_base + kOffBars;
+    const uint32_t bar_full = smem_base + kOffBars, bar_empty = bar_full + kStages * 8;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_full + s * 8, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + s * 8, 1);
+            mbar_init(bar_empty + s * 8, kConsumerWarps);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -91,9 +99,11 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
         c_it = item_at(item_lo);
         c_tile = c_it.tile_begin;
     }
-    auto issue_next_tile = [&]() {  // thread 0 only; the stage it writes must be free
+    auto issue_next_tile = [&]() {  // thread 0 only
         if (c_item >= item_hi) return;
         const uint32_t s = c_fill % kStages;
+        // the stage is free when all eight warps have released the tile that used it last
+        if (!mbar_wait(bar_empty + s * 8, ((c_fill / kStages) & 1) ^ 1, abort_flag, p.error_flag, 21)) return;
         const int rows = min(T, (c_it.kv_end - c_tile * T + 15) & ~15);  // 16-token steps that hold visible tokens
         mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
         const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
@@ -198,8 +208,8 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                 mxs[ch * kRows + rb * 16 + g8] = mx0;
                 mxs[ch * kRows + rb * 16 + g8 + 8] = mx1;
             }
-            consumer_bar();  // (1) both halves' row maxima are visible; every warp is done with the tile before this one
-            if (tid == 0) issue_next_tile();  // ... so its stage takes the tile after this one
+            pair_bar(rb);  // (1) both halves' row maxima are visible
+            if (tid == 0) issue_next_tile();  // the tile after this one, into the stage of the tile before it
 
             // ---- running max, weights of this half, exchange of the bf16 weight tile ----
             mx0 = fmaxf(mxs[rb * 16 + g8], mxs[kRows + rb * 16 + g8]);
@@ -232,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                     o[n][3] *= a1;
                 }
             }
-            consumer_bar();  // (2) the weight tile is complete
+            pair_bar(rb);  // (2) the weight tile is complete
 
             // ---- O[16 rows, 256 latent columns] += P[16 x 64] . C[64 x 256] ----
             if (live) {
@@ -266,6 +276,8 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
                     }
                 }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + s_idx * 8);  // this warp is done with the stage
         }
 
         // ---- end of the item: row sums of the two halves, then the result ----
@@ -277,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
             sums[ch * kRows + rb * 16 + g8] = l[0];
             sums[ch * kRows + rb * 16 + g8 + 8] = l[1];
         }
-        consumer_bar();
+        pair_bar(rb);
         const float lt0 = sums[rb * 16 + g8] + sums[kRows + rb * 16 + g8];
         const float lt1 = sums[rb * 16 + g8 + 8] + sums[kRows + rb * 16 + g8 + 8];
         const float inv0 = lt0 > 0.f ? 1.f / lt0 : 0.f, inv1 = lt1 > 0.f ? 1.f / lt1 : 0.f;

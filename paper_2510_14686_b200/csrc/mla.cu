@@ -7,15 +7,15 @@
 // lands in shared memory with nine linear bulk copies and feeds ldmatrix without bank conflicts, as in the GQA kernel.
 //
 // One persistent CTA per SM (8 warps, 255 registers per thread) walks its run of work items (64 heads of one query
-// token x a range of tiles).  Tiles arrive in a two-stage ring (cp.async.bulk + mbarrier transaction counts); one
-// elected thread issues the copy of tile f+1 right after the CTA-wide barrier in the middle of tile f, which every
-// warp reaches only when it is done with tile f-1, so the stage is free without a second set of barriers.  (A ninth,
-// copy-only warp would cap the kernel at 168 registers per thread: the register file is allocated as if the CTA had
-// 384 threads.)  Warp (rb, ch) owns rows
+// token x a range of tiles).  Tiles arrive in a two-stage ring (cp.async.bulk + mbarrier transaction counts, released
+// per warp through a second set of mbarriers); one elected thread issues the copy of tile f+1 in the middle of tile f.
+// (A ninth, copy-only warp would cap the kernel at 168 registers per thread: the register file is allocated as if the
+// CTA had 384 threads.)  Warp (rb, ch) owns rows
 // 16 rb..16 rb+15; for Q.K^T it takes tokens 32 ch..32 ch+31 of the tile over all 576 dims (Q fragments come from
 // shared memory, they do not fit registers), the two halves agree on row maxima through shared memory and exchange
-// their bf16 weights, and for P.V the warp accumulates all 64 tokens into latent columns 256 ch..256 ch+255
-// (128 fp32 registers per thread).  The contraction runs on mma.sync m16n8k16: with 128 heads per token this path is
+// their bf16 weights (the two warps of a row block synchronise with a 64-thread barrier of their own, so the four row
+// blocks drift apart and mix their load- and MMA-heavy phases), and for P.V the warp accumulates all 64 tokens into
+// latent columns 256 ch..256 ch+255 (128 fp32 registers per thread).  The contraction runs on mma.sync m16n8k16: with 128 heads per token this path is
 // as much tensor- as HBM-bound, and a tcgen05/TMEM version of the two contractions is the step after this one.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>

@@ -176,3 +176,41 @@ def test_modes_refuse_each_others_calls(binding):
         assert e.value.status == binding.ERR_UNSUPPORTED
     with pytest.raises(binding.XllmError):             # wrong geometry for the flag
         binding.Context(100, 1, D, 1, 256, 4 * PAGE, flags=binding.FLAG_MLA)
+
+
+@pytest.mark.parametrize("name", ["decode", "verify"])
+def test_bench_sized_batch_on_sampled_rows(binding, name):
+    """The side benchmark's batch shape (lengths, heads, q_len) at full size; the oracle checks sampled (row, head) pairs."""
+    from gpu_harness import dev_bits, host_bits
+
+    kv, ql = wl.mla_lengths(name)
+    H = wl.MLA_HEADS
+    gen = torch.Generator().manual_seed(4000 + len(kv))
+    rows = int(ql.sum())
+    q = wl.bf16_bits(torch.randn(rows, H, D, generator=gen) * 0.25)
+    with mla_ctx(binding, H, len(kv), int(kv.max()) + 64, kv, max_q_len=int(ql.max())) as ctx:
+        slots, caches = [], {}
+        sampled = sorted(set(int(x) for x in np.random.default_rng(5).integers(0, len(kv), 6)) | {int(np.argmax(kv)), int(np.argmin(kv))})
+        for r, n in enumerate(kv):
+            c = wl.bf16_bits(torch.randn(int(n), D, generator=gen))
+            s = ctx.kv_reserve(expected_tokens=int(n))
+            ctx.kv_map_pages(s, int(n))
+            ctx.mla_append([s], [int(n)], dev_bits(c))
+            slots.append(s)
+            if r in sampled:
+                caches[r] = c
+        out = torch.zeros((rows, H, wl.MLA_D_C), dtype=torch.int16, device="cuda")
+        lse = torch.zeros((rows, H), dtype=torch.float32, device="cuda")
+        scale = 1.0 / float(np.sqrt(128 + wl.MLA_D_R))
+        ctx.mla_attention(slots, dev_bits(q), out, lse, None if int(ql.max()) == 1 else ql, scale)
+        ctx.sync_check()
+        got, got_lse = wl.bits_to_f64(host_bits(out)), lse.cpu().numpy()
+    assert np.isfinite(got).all()
+    row0 = np.concatenate([[0], np.cumsum(ql)])
+    heads = [0, 17, 63, 64, 127]
+    for r in sampled:
+        rr = slice(int(row0[r]), int(row0[r + 1]))
+        ref_o, ref_l = mla_oracle.mla_attention(q[rr][:, heads], caches[r], scale, wl.MLA_D_C)
+        err = np.abs(got[rr][:, heads] - ref_o)
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (r, err.max(), err.mean())
+        assert np.abs(got_lse[rr][:, heads] - ref_l).max() <= LSE_ABS

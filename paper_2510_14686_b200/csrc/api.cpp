@@ -60,6 +60,7 @@ struct GraphStep {
 };
 
 struct xllm_ctx {
+    bool mla_tcgen05 = false;  // MLA: scores on tcgen05 + tensor memory (XLLM_MLA_KERNEL=tcgen05) instead of mma.sync
     bool mla = false;  // XLLM_FLAG_MLA: slots hold one 576-dim latent vector per token; only the xllm_mla_* calls compute on them
     std::vector<int64_t> mla_kv;      // per query token of an MLA call: keys it sees
     std::vector<int32_t> mla_req;     // ... and the request it belongs to
@@ -526,6 +527,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     ctx->cfg = *cfg;
     ctx->host_only = (cfg->flags & XLLM_FLAG_HOST_ONLY) != 0;
     ctx->mla = mla;
+    if (const char *k = std::getenv("XLLM_MLA_KERNEL")) ctx->mla_tcgen05 = std::string(k) == "tcgen05";
     const int64_t row_bytes = mla ? (int64_t)kMlaDim * 2 : 2ll * cfg->n_kv_heads * cfg->head_dim * 2;
     std::unique_ptr<VmmDriver> drv;
     if (ctx->host_only) {
@@ -1213,7 +1215,7 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ml.n_ctas = ctx->sm_count;
     std::memcpy(ml.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
     time_begin(ctx, 0, stream);
-    e = launch_mla_attention(ml, stream);
+    e = launch_mla_attention(ml, ctx->mla_tcgen05, stream);
     time_end(ctx, stream);
     if (e) return cuda_fail(ctx, "launching the latent attention kernel", e);
     ++ctx->st.kernel_launches;

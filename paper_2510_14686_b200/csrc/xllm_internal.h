@@ -211,7 +211,7 @@ int launch_gather(uint64_t base, int64_t first_token, int64_t n_tokens, void *k_
 
 // mla.cu
 int mla_configure_kernels();
-int launch_mla_attention(const MlaLaunch &p, void *stream);
+int launch_mla_attention(const MlaLaunch &p, bool scores_on_tcgen05, void *stream);
 int launch_mla_combine(const CombineDesc *descs, int32_t n_units, const float *part_o, const float *part_lse, void *out,
                        float *lse_out, int32_t n_heads, void *stream);
 int launch_mla_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const void *c_new, void *stream);

@@ -1210,6 +1210,7 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ml.comb_src = reinterpret_cast<const CombineDesc *>(d + off_comb);
     ml.comb_dst = ctx->d_mla_comb;
     ml.n_comb = (int32_t)combine.size();
+    ml.trace = ctx->d_trace;
     ml.n_heads = ctx->cfg.n_q_heads;
     ml.scale_log2 = scale * 1.4426950408889634f;
     ml.n_ctas = ctx->sm_count;

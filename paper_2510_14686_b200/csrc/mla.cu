@@ -483,9 +483,12 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
     const bool sm_warp = rb < 2;                // this warp's lane quarter of tensor memory holds real rows
     const int sm_row = rb * 32 + lane;          // ... and this thread reads row sm_row, columns 32 ch .. 32 ch + 31
     bool live = true;
+    const bool tr = p.trace != nullptr;
+    unsigned long long t_all = tr ? clock64() : 0ull, t_wait_s = 0, t_softmax = 0, t_wait_a = 0, t_pv = 0, t_wait_b = 0, t_item = 0, t_post = 0, n_tiles = 0;
 
     for (int i = item_lo; i < item_hi; ++i) {
         const MlaItem it = item_at(i);
+        unsigned long long t0 = tr ? clock64() : 0ull;
         __syncthreads();  // everybody is done with the previous item's query rows (its last scores were read long ago)
         {
             const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.q) +
@@ -508,6 +511,7 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
 #pragma unroll
         for (int n = 0; n < kDv / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
         float m_run = -INFINITY, l_run = 0.f;  // softmax threads: state of row sm_row (the sum over this thread's columns only)
+        if (tr) t_item += clock64() - t0;
 
         for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
             const uint32_t s_idx = fill % kStages, ph = (fill / kStages) & 1;
@@ -516,8 +520,10 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
             const bool tail = tile_tok0 + T > it.kv_end;
 
             // ---- softmax of the tile: one row per thread ----
+            if (tr) t0 = clock64(), ++n_tiles;
             if (sm_warp) {
                 live = __all_sync(0xffffffffu, mbar_wait(bar_sdone + (fill & 1u) * 8, ph, abort_flag, p.error_flag, 23)) && live;
+                if (tr) t_wait_s += clock64() - t0, t0 = clock64();
                 float sv[32];
                 if (live) {
                     tc_fence_after();
@@ -552,8 +558,10 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
 #pragma unroll
                 for (int j = 0; j < 4; ++j) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
                 if (ch == 0) corr_s[sm_row] = a;
+                if (tr) t_softmax += clock64() - t0, t0 = clock64();
             }
             __syncthreads();  // (A) weights and correction factors of the tile are visible
+            if (tr) t_wait_a += clock64() - t0, t0 = clock64();
 
             // ---- rescale, then O[16 rows, 256 latent columns] += P[16 x 64] . C[64 x 256] on mma.sync ----
             const float a0 = corr_s[rb * 16 + g8], a1 = corr_s[rb * 16 + g8 + 8];
@@ -603,11 +611,16 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
                     }
                 }
             }
-            if (tid == 0 && more && s_issued <= fill + 1) {  // not landed while the steps ran: wait for it (bounded)
-                if (mbar_wait(bar_full + ((fill + 1) % kStages) * 8, ((fill + 1) / kStages) & 1, abort_flag, p.error_flag, 25)) issue_scores(fill + 1);
-            }
+            if (tr) t_pv += clock64() - t0, t0 = clock64();
             __syncthreads();  // (B) everybody is done with the weight tile and with this stage
-            if (tid == 0) issue_next_copy();  // the tile two ahead, into the stage just freed
+            if (tr) t_wait_b += clock64() - t0, t0 = clock64();
+            if (tid == 0) {
+                issue_next_copy();  // the tile two ahead, into the stage just freed (first: the copies must never wait for one another)
+                if (more && s_issued <= fill + 1) {  // the next tile had not landed while the steps ran: wait for it (bounded)
+                    if (mbar_wait(bar_full + ((fill + 1) % kStages) * 8, ((fill + 1) / kStages) & 1, abort_flag, p.error_flag, 25)) issue_scores(fill + 1);
+                }
+                if (tr) t_post += clock64() - t0;
+            }
         }
 
         // ---- end of the item: row sums and maxima from the softmax threads, then the result ----
@@ -648,6 +661,10 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
                 }
             }
         }
+    }
+    if (tr && lane == 0 && (warp == 0 || warp == 2)) {
+        unsigned long long *w = p.trace + (size_t)blockIdx.x * kTraceWords + (warp == 0 ? 0 : 8);
+        w[0] = clock64() - t_all, w[1] = n_tiles, w[2] = t_wait_s, w[3] = t_softmax, w[4] = t_wait_a, w[5] = t_pv, w[6] = t_wait_b, w[7] = warp == 0 ? t_post : t_item;
     }
     // A wait ran out: give the copies and the MMAs still in flight a bounded time to finish before the CTA gives up its
     // shared and tensor memory.

@@ -148,6 +148,9 @@ xllm_status check_device_flag(xllm_ctx *ctx) {
         cudaDeviceSynchronize();
         if (ctx->d_counters) cudaMemset(ctx->d_counters, 0, sizeof(int32_t) * ((size_t)ctx->max_partials + 1));
         ctx->pool_base = 0;
+        if (code == 30)
+            return fail(ctx, XLLM_ERR_CUDA, "attention kernel: shared memory of the CTA is not 1 KiB aligned, which the tensor-core matrix "
+                                            "descriptors need (code 30); the launch did nothing");
         return fail(ctx, XLLM_ERR_CUDA, "attention kernel: a bounded device-side wait expired (code " + std::to_string(code) +
                                             "); the results of that launch are invalid");
     }
@@ -1210,11 +1213,16 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ml.comb_src = reinterpret_cast<const CombineDesc *>(d + off_comb);
     ml.comb_dst = ctx->d_mla_comb;
     ml.n_comb = (int32_t)combine.size();
-    ml.trace = ctx->d_trace;
     ml.n_heads = ctx->cfg.n_q_heads;
     ml.scale_log2 = scale * 1.4426950408889634f;
     ml.n_ctas = ctx->sm_count;
     std::memcpy(ml.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    ml.debug_stall_cta = -1;
+    if (ctx->inject_timeouts > 0) {
+        --ctx->inject_timeouts;
+        for (int32_t c = 0; c < ctx->sm_count; ++c)
+            if (ml.cta_begin[c] < ml.cta_begin[c + 1]) { ml.debug_stall_cta = c; break; }
+    }
     time_begin(ctx, 0, stream);
     e = launch_mla_attention(ml, ctx->mla_tcgen05, stream);
     time_end(ctx, stream);

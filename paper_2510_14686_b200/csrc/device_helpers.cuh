@@ -56,7 +56,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // skip their work but keep executing the barrier protocol so that no warp is left waiting.
 // (the waiting loop is kept out of line: the kernel has some twenty waits, most of them in its hottest loops, and the
 // instruction cache is a scarce resource here)
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
+__device__ __forceinline__ bool mbar_wait_loop(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
@@ -70,11 +70,21 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         }
     }
 }
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
+    return mbar_wait_loop(bar, parity, abort_flag, error_flag, code);
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag,
                                           int code) {
     if (*abort_flag) return false;
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, error_flag, code);
+}
+// The same with the loop in line, for kernels that change their register budget per warp (setmaxnreg): the assembler
+// cannot allocate registers across a call there.
+__device__ __forceinline__ bool mbar_wait_inl(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *error_flag, int code) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_loop(bar, parity, abort_flag, error_flag, code);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),

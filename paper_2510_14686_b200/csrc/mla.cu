@@ -108,8 +108,10 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
         mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
         const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
         const char *src = reinterpret_cast<const char *>(c_it.kv) + (int64_t)c_tile * kTileBytes;
+        const int n_copy = ((int)blockIdx.x == p.debug_stall_cta && c_fill == 0) ? kPanels - 1 : kPanels;  // test hook: the wait on this tile must run out
 #pragma unroll
-        for (int pn = 0; pn < kPanels; ++pn) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
+        for (int pn = 0; pn < kPanels; ++pn)
+            if (pn < n_copy) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
         ++c_fill;
         if (++c_tile >= c_it.tile_end) {
             if (++c_item < item_hi) {
@@ -335,22 +337,35 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel(const __grid
     __syncthreads();
 }
 
-// ---- the same work with Q.K^T on the 5th-generation tensor cores -----------------------------------------------
+// ---- the same work, warp-specialised, with Q.K^T on the 5th-generation tensor cores -------------------------------
 // S = Q.K^T is a plain dense contraction whose operands already sit in shared memory in the canonical K-major
 // 128-byte-swizzled form (a panel row is 64 dims = 128 bytes, chunks XOR-ed by row & 7, panels 1 KiB aligned): one
 // thread issues it as 36 tcgen05.mma (M 128 x N 64 x K 16, bf16 -> fp32) straight from shared-memory descriptors into
-// tensor memory, no fragment loads at all.  The item has 64 heads, so rows 64..127 of the MMA read whatever follows the
-// query panel (in bounds) and their results are never looked at.  Four warps (the ones whose lane quarter holds real
-// rows) read the scores back with tcgen05.ld, one row per thread: row maximum, weights and sums need no shuffles.  The
-// bf16 weights go to shared memory, and P.V stays on mma.sync with the output in registers as above: the accumulator
-// of 64 heads x 512 columns would fill tensor memory on its own.  S of tile f+1 runs on the tensor cores while the
-// warps do P.V of tile f.
+// tensor memory, with no fragment loads at all.  The item has 64 heads, so rows 64..127 of the MMA read whatever
+// follows the query panel (in bounds) and their results are never looked at.  Twelve warps:
+//   0-7   P.V on mma.sync with the output in registers (the accumulator of 64 heads x 512 columns would fill tensor
+//         memory on its own), exactly as in the kernel above;
+//   8-9   softmax: the two warps whose lane quarter of tensor memory holds real rows read the scores back with
+//         tcgen05.ld, one whole row per thread, so maxima, weights and sums need no exchange at all; they write the bf16
+//         weights into panel 8 of the tile's own stage (the rotary dims, dead once the scores exist: the weight tile is
+//         double-buffered for free) and the factor by which each row's maximum moved; they also bring in the query rows
+//         of the next item when the scores of the last tile of the current one exist;
+//   10    one lane issues the score MMAs, one tile ahead of the softmax (two score buffers in tensor memory);
+//   11    (the last warp) one lane issues the tile copies as soon as the P.V warps release a stage.
+// Everything is handed over through mbarriers (bounded waits), so scores, softmax and copies of tiles f+1, f+2 run under
+// P.V of tile f.
 namespace tc {
-constexpr int kOffCorr = kOffMx + 2 * kRows * 4;                 // [64] factor by which a row's running maximum moved
-constexpr int kOffM = kOffCorr + kRows * 4;                      // [64] running maximum at the end of the item
-constexpr int kOffBars = kOffM + kRows * 4;                      // full[kStages], sdone[2]
-constexpr int kOffFlags = kOffBars + (kStages + 2) * 8;          // [0] abort flag, [1] tensor-memory base
-constexpr int kItemCache = 14;
+constexpr int kPvWarps = 8;
+constexpr int kSoftmaxWarp0 = 8;
+constexpr int kMmaWarp = 10;
+constexpr int kThreadsWs = 12 * 32;
+constexpr int kOffCorr = kOffKV + kStages * kTileBytes;          // [2][64] factor by which a row's running maximum moved (per tile parity)
+constexpr int kOffLsum = kOffCorr + 2 * kRows * 4;               // [2][64] row sums at the end of an item (per item parity)
+constexpr int kOffMfin = kOffLsum + 2 * kRows * 4;               // [2][64] row maxima at the end of an item
+constexpr int kOffBars = kOffMfin + 2 * kRows * 4;               // full, sdone, sfree, pready, stfree, fin: two of each
+constexpr int kNumBars = 12;
+constexpr int kOffFlags = kOffBars + kNumBars * 8;               // [0] abort flag, [1] tensor-memory base
+constexpr int kItemCache = 32;
 constexpr int kOffItems = kOffFlags + 16;
 constexpr int kSmemBytes = kOffItems + kItemCache * (int)sizeof(MlaItem);
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
@@ -371,7 +386,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {  // 32 consecutive columns of this thread's lane
     uint32_t r[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,"
@@ -389,25 +404,36 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 }  // namespace tc
 
-__global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __grid_constant__ MlaLaunch p) {
+__global__ void __launch_bounds__(tc::kThreadsWs, 1) mla_attention_kernel_tc(const __grid_constant__ MlaLaunch p) {
     using namespace tc;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + tc::kOffFlags);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + tc::kOffFlags + 4);
-    const uint32_t bar_full = smem_base + tc::kOffBars, bar_sdone = bar_full + kStages * 8;
+    const uint32_t bar_full = smem_base + tc::kOffBars;  // [2] tile landed (copy -> MMA lane, P.V warps)
+    const uint32_t bar_sdone = bar_full + 16;            // [2] scores of a tile complete (MMA -> softmax)
+    const uint32_t bar_sfree = bar_full + 32;            // [2] score buffer read out (softmax -> MMA lane)
+    const uint32_t bar_pready = bar_full + 48;           // [2] weights and factors of a tile written (softmax -> P.V)
+    const uint32_t bar_stfree = bar_full + 64;           // [2] stage (and its weights and factors) no longer needed (P.V -> copy lane)
+    const uint32_t bar_fin = bar_full + 80;              // [2] row sums and maxima of an item written (softmax -> P.V)
     if (smem_base & 1023u) {  // the swizzle of the matrix descriptors is a function of the address: panels must be 1 KiB aligned
         if (tid == 0) *reinterpret_cast<volatile int32_t *>(p.error_flag) = 30;
         return;
     }
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_full + s * 8, 1);
-        for (int b = 0; b < 2; ++b) mbar_init(bar_sdone + b * 8, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_full + b * 8, 1);
+            mbar_init(bar_sdone + b * 8, 1);
+            mbar_init(bar_sfree + b * 8, 2);
+            mbar_init(bar_pready + b * 8, 2);
+            mbar_init(bar_stfree + b * 8, kPvWarps);
+            mbar_init(bar_fin + b * 8, 2);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {  // one warp allocates (and at the end frees) the tensor memory of the CTA
+    if (warp == kMmaWarp) {  // this warp allocates (and at the end frees) the tensor memory of the CTA
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + tc::kOffFlags + 4), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -423,268 +449,261 @@ __global__ void __launch_bounds__(kThreads, 1) mla_attention_kernel_tc(const __g
     grid_launch_dependents();
     grid_dependency_wait();  // the previous kernel of the stream may still write q or the slots
     auto item_at = [&](int i) -> MlaItem { return (i - item_lo < tc::kItemCache) ? sitems[i - item_lo] : p.items[i]; };
-    for (int i = blockIdx.x * kThreads + tid; i < p.n_comb * (int)(sizeof(CombineDesc) / 8); i += p.n_ctas * kThreads)
+    for (int i = blockIdx.x * kThreadsWs + tid; i < p.n_comb * (int)(sizeof(CombineDesc) / 8); i += p.n_ctas * kThreadsWs)
         reinterpret_cast<uint2 *>(p.comb_dst)[i] = reinterpret_cast<const uint2 *>(p.comb_src)[i];
 
-    uint32_t fill = 0;  // tiles of this CTA so far: stage = fill % kStages, score buffer = fill % 2, use = fill / 2
-
-    // ---- thread 0: copies run up to two tiles ahead of the computation; the scores of a tile are issued one tile ahead ----
-    int c_item = item_lo, c_tile = 0;
-    uint32_t c_fill = 0;
-    MlaItem c_it = {};
-    if (tid == 0 && item_lo < item_hi) {
-        c_it = item_at(item_lo);
-        c_tile = c_it.tile_begin;
-    }
-    auto issue_next_copy = [&]() {  // thread 0 only; the stage it writes must be free
-        if (c_item >= item_hi) return;
-        const uint32_t s = c_fill % kStages;
-        const int rows = min(T, (c_it.kv_end - c_tile * T + 15) & ~15);  // 16-token steps that hold visible tokens
-        mbar_expect_tx(bar_full + s * 8, kPanels * rows * 128);
-        const uint32_t dst = smem_base + kOffKV + s * kTileBytes;
-        const char *src = reinterpret_cast<const char *>(c_it.kv) + (int64_t)c_tile * kTileBytes;
-#pragma unroll
-        for (int pn = 0; pn < kPanels; ++pn) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + s * 8);
-        ++c_fill;
-        if (++c_tile >= c_it.tile_end) {
-            if (++c_item < item_hi) {
-                c_it = item_at(c_item);
-                c_tile = c_it.tile_begin;
-            }
-        }
-    };
-    uint32_t s_issued = 0;  // (thread 0) the scores of tiles [0, s_issued) of this CTA have been issued
-    auto issue_scores = [&](uint32_t f) {  // thread 0 only: S(tile f) = Q . K^T into score buffer f % 2; the tile has landed
-        tc_fence_after();
-        const uint64_t adesc = kDescHi | (uint64_t)((smem_base + kOffQ) >> 4);
-        const uint64_t bdesc = kDescHi | (uint64_t)((smem_base + kOffKV + (f % kStages) * kTileBytes) >> 4);
-        const uint32_t d = tmem_base + (f & 1u) * 64u;
-#pragma unroll
-        for (int pn = 0; pn < kPanels; ++pn)
-#pragma unroll
-            for (int k16 = 0; k16 < 4; ++k16) {
-                const uint64_t off = (uint64_t)((pn * kPanelBytes + k16 * 32) >> 4);
-                umma_bf16(d, adesc + off, bdesc + off, (pn | k16) ? 1u : 0u);
-            }
-        umma_commit(bar_sdone + (f & 1u) * 8);
-        s_issued = f + 1;
-    };
-    if (tid == 0) {
-        issue_next_copy();
-        issue_next_copy();
-    }
-
-    const int rb = warp & 3, ch = warp >> 2;
-    const int g8 = lane >> 2, q4 = lane & 3, swz = lane & 7;
-    float *mxs = reinterpret_cast<float *>(smem + kOffMx);
     float *corr_s = reinterpret_cast<float *>(smem + tc::kOffCorr);
-    float *m_s = reinterpret_cast<float *>(smem + tc::kOffM);
-    const uint32_t p_smem = smem_base + kOffP;
-    const bool sm_warp = rb < 2;                // this warp's lane quarter of tensor memory holds real rows
-    const int sm_row = rb * 32 + lane;          // ... and this thread reads row sm_row, columns 32 ch .. 32 ch + 31
-    bool live = true;
-    const bool tr = p.trace != nullptr;
-    unsigned long long t_all = tr ? clock64() : 0ull, t_wait_s = 0, t_softmax = 0, t_wait_a = 0, t_pv = 0, t_wait_b = 0, t_item = 0, t_post = 0, n_tiles = 0;
+    float *lsum_s = reinterpret_cast<float *>(smem + tc::kOffLsum);
+    float *mfin_s = reinterpret_cast<float *>(smem + tc::kOffMfin);
+    uint32_t f = 0;  // tiles of this CTA so far (every role counts them the same way): stage = score buffer = f & 1, use = f >> 1
 
-    for (int i = item_lo; i < item_hi; ++i) {
-        const MlaItem it = item_at(i);
-        unsigned long long t0 = tr ? clock64() : 0ull;
-        __syncthreads();  // everybody is done with the previous item's query rows (its last scores were read long ago)
-        {
-            const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.q) +
-                                                               ((int64_t)it.q_row * p.n_heads + it.head0) * (kD * 2));
-            constexpr int kChunks = kRows * (kD / 8);
-#pragma unroll 6
-            for (int c = tid; c < kChunks; c += kThreads) {
-                const int r = c / (kD / 8), cc = c % (kD / 8);
-                const uint4 v = src[c];
-                *reinterpret_cast<uint4 *>(smem + kOffQ + (cc >> 3) * kPanelBytes + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = v;
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores before the tensor cores read them
-        }
-        __syncthreads();
-        if (tid == 0) {  // scores of the item's first tile
-            if (mbar_wait(bar_full + (fill % kStages) * 8, (fill / kStages) & 1, abort_flag, p.error_flag, 22)) issue_scores(fill);
-        }
-
-        float o[kDv / 2 / 8][4];
+    if (warp < kPvWarps) {
+        // ================= P.V warps =================
+        const int rb = warp & 3, ch = warp >> 2;
+        const int g8 = lane >> 2, q4 = lane & 3, swz = lane & 7;
+        const int r0 = rb * 16 + g8, r1 = r0 + 8;
+        bool live = true;
+        uint32_t n_item = 0;
+        for (int i = item_lo; i < item_hi; ++i, ++n_item) {
+            const MlaItem it = item_at(i);
+            float o[kDv / 2 / 8][4];
 #pragma unroll
-        for (int n = 0; n < kDv / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;  // softmax threads: state of row sm_row (the sum over this thread's columns only)
-        if (tr) t_item += clock64() - t0;
-
-        for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++fill) {
-            const uint32_t s_idx = fill % kStages, ph = (fill / kStages) & 1;
-            const uint32_t stage = smem_base + kOffKV + s_idx * kTileBytes;
-            const int tile_tok0 = tile * T;
-            const bool tail = tile_tok0 + T > it.kv_end;
-
-            // ---- softmax of the tile: one row per thread ----
-            if (tr) t0 = clock64(), ++n_tiles;
-            if (sm_warp) {
-                live = __all_sync(0xffffffffu, mbar_wait(bar_sdone + (fill & 1u) * 8, ph, abort_flag, p.error_flag, 23)) && live;
-                if (tr) t_wait_s += clock64() - t0, t0 = clock64();
-                float sv[32];
+            for (int n = 0; n < kDv / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+            float lt0 = 0.f, lt1 = 0.f, m0 = -INFINITY, m1 = -INFINITY;
+            for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++f) {
+                const uint32_t b = f & 1u, ph = (f >> 1) & 1u;
+                const uint32_t stage = smem_base + kOffKV + b * kTileBytes;
+                const int tile_tok0 = tile * T;
+                const bool tail = tile_tok0 + T > it.kv_end;
+                live = __all_sync(0xffffffffu, mbar_wait_inl(bar_pready + b * 8, ph, abort_flag, p.error_flag, 35)) && live;
+                live = __all_sync(0xffffffffu, mbar_wait_inl(bar_full + b * 8, ph, abort_flag, p.error_flag, 36)) && live;  // (landed long ago; the wait makes the copy visible to this thread)
+                const float a0 = corr_s[b * kRows + r0], a1 = corr_s[b * kRows + r1];
+                if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {  // the running maximum moved: rescale the accumulator
+#pragma unroll
+                    for (int n = 0; n < kDv / 16; ++n) {
+                        o[n][0] *= a0;
+                        o[n][1] *= a0;
+                        o[n][2] *= a1;
+                        o[n][3] *= a1;
+                    }
+                }
+                if (live) {
+                    const int n_ks = tail ? min(4, (it.kv_end - tile_tok0 + 15) >> 4) : 4;  // 16-token steps that were fetched
+                    const uint32_t p_row = stage + 8 * kPanelBytes + (rb * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * 128;
+                    const int vr = (lane & 7) + (((lane >> 3) & 1) << 3);
+                    const int v_csel = lane >> 4;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        if (kk >= n_ks) break;
+                        uint32_t pa[4];
+                        ldsm_x4(pa[0], pa[1], pa[2], pa[3], p_row + (((2 * kk + v_csel) ^ swz) << 4));
+                        uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
+                        if (tail) {  // rows never written may hold anything: force them to zero (0 * NaN would poison O)
+                            const int t0 = tile_tok0 + kk * 16 + 2 * q4;
+                            vmask0 = (t0 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < it.kv_end ? 0xffff0000u : 0u);
+                            vmask1 = (t0 + 8 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < it.kv_end ? 0xffff0000u : 0u);
+                        }
+                        const uint32_t row_addr = stage + (kk * 16 + vr) * 128;
+#pragma unroll
+                        for (int n2 = 0; n2 < kDv / 32; ++n2) {
+                            const int cg = ch * (kDv / 16) + 2 * n2 + v_csel;  // 8-column chunk of the latent dims
+                            uint32_t b0, b1, b2, b3;
+                            ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
+                            b0 &= vmask0;
+                            b1 &= vmask1;
+                            b2 &= vmask0;
+                            b3 &= vmask1;
+                            mma_bf16(o[2 * n2], pa, b0, b1);
+                            mma_bf16(o[2 * n2 + 1], pa, b2, b3);
+                        }
+                    }
+                }
+                if (tile + 1 == it.tile_end) {
+                    // the item's row sums and maxima: read before the last stage goes back, which is what keeps the softmax
+                    // warps from overwriting them two items later
+                    live = __all_sync(0xffffffffu, mbar_wait_inl(bar_fin + (n_item & 1u) * 8, (n_item >> 1) & 1u, abort_flag, p.error_flag, 37)) && live;
+                    lt0 = lsum_s[(n_item & 1u) * kRows + r0];
+                    lt1 = lsum_s[(n_item & 1u) * kRows + r1];
+                    m0 = mfin_s[(n_item & 1u) * kRows + r0];
+                    m1 = mfin_s[(n_item & 1u) * kRows + r1];
+                }
+                // (every ldmatrix above has fed an MMA that was issued before this point: the loads have delivered)
+                __syncwarp();
+                if (lane == 0) mbar_arrive_after(bar_stfree + b * 8, __float_as_uint(lt0) ^ __float_as_uint(m1) ^ __float_as_uint(a0), smem_base + tc::kOffFlags + 8);
+            }
+            const float inv0 = lt0 > 0.f ? 1.f / lt0 : 0.f, inv1 = lt1 > 0.f ? 1.f / lt1 : 0.f;
+            if (live) {
+                if (it.partial_idx < 0) {
+                    __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.out);
+                    const int64_t base0 = ((int64_t)it.q_row * p.n_heads + it.head0 + r0) * kDv + ch * (kDv / 2) + 2 * q4;
+                    const int64_t base1 = base0 + 8ll * kDv;
+#pragma unroll
+                    for (int n = 0; n < kDv / 16; ++n) {
+                        *reinterpret_cast<uint32_t *>(out + base0 + n * 8) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
+                        *reinterpret_cast<uint32_t *>(out + base1 + n * 8) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
+                    }
+                    if (p.lse_out && ch == 0 && q4 == 0) {  // natural log
+                        p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r0] = lt0 > 0.f ? m0 * 0.6931471805599453f + logf(lt0) : -INFINITY;
+                        p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r1] = lt1 > 0.f ? m1 * 0.6931471805599453f + logf(lt1) : -INFINITY;
+                    }
+                } else {
+                    float *po = p.part_o + (int64_t)it.partial_idx * kRows * kDv;
+                    const int64_t base0 = (int64_t)r0 * kDv + ch * (kDv / 2) + 2 * q4, base1 = base0 + 8ll * kDv;
+#pragma unroll
+                    for (int n = 0; n < kDv / 16; ++n) {
+                        *reinterpret_cast<float2 *>(po + base0 + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+                        *reinterpret_cast<float2 *>(po + base1 + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+                    }
+                    if (ch == 0 && q4 == 0) {  // log2 domain
+                        p.part_lse[(int64_t)it.partial_idx * kRows + r0] = lt0 > 0.f ? m0 + log2f(lt0) : -INFINITY;
+                        p.part_lse[(int64_t)it.partial_idx * kRows + r1] = lt1 > 0.f ? m1 + log2f(lt1) : -INFINITY;
+                    }
+                }
+            }
+        }
+    } else {
+      if (warp < kMmaWarp) {
+        // ================= softmax warps: thread = one row of the item =================
+        const int row = (warp - kSoftmaxWarp0) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;  // this warp's quarter of the tensor-memory lanes
+        bool live = true;
+        uint32_t n_item = 0;
+        for (int i = item_lo; i < item_hi; ++i, ++n_item) {
+            const MlaItem it = item_at(i);
+            {
+                // Query rows of the item's 64 heads -> swizzled panels.  The score MMAs of the previous item are complete:
+                // these warps have waited for the last of them.
+                const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(p.q) +
+                                                                   ((int64_t)it.q_row * p.n_heads + it.head0) * (kD * 2));
+                constexpr int kChunks = kRows * (kD / 8);  // 4608 chunks of 16 bytes: 72 per thread
+#pragma unroll 8
+                for (int c = tid - kSoftmaxWarp0 * 32; c < kChunks; c += 64) {
+                    const int r = c / (kD / 8), cc = c % (kD / 8);
+                    const uint4 v = src[c];
+                    *reinterpret_cast<uint4 *>(smem + kOffQ + (cc >> 3) * kPanelBytes + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = v;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy stores before the tensor cores read them
+                __syncwarp();
+                asm volatile("bar.sync 1, 96;" ::: "memory");  // with the MMA warp: the query panels are in place
+            }
+            float m_run = -INFINITY, l_run = 0.f;
+            for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++f) {
+                const uint32_t b = f & 1u, ph = (f >> 1) & 1u;
+                const int tile_tok0 = tile * T;
+                const bool tail = tile_tok0 + T > it.kv_end;
+                live = __all_sync(0xffffffffu, mbar_wait_inl(bar_sdone + b * 8, ph, abort_flag, p.error_flag, 34)) && live;
+                float sv[T];  // one row, 64 columns
                 if (live) {
                     tc_fence_after();
-                    tmem_ld32(tmem_base + ((uint32_t)(rb * 32) << 16) + (fill & 1u) * 64u + ch * 32u, sv);
+                    tmem_ld32(tmem_base + lane_base + b * 64u, sv);
+                    tmem_ld32(tmem_base + lane_base + b * 64u + 32u, sv + 32);
                     tc_fence_before();
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) sv[j] = -INFINITY;
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive_after(bar_sfree + b * 8, __float_as_uint(sv[0]) ^ __float_as_uint(sv[63]), smem_base + tc::kOffFlags + 12);
                 float mx = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    sv[j] = (!tail || tile_tok0 + ch * 32 + j < it.kv_end) ? sv[j] * p.scale_log2 : -INFINITY;  // (also drops NaN of stale rows)
+                for (int j = 0; j < T; ++j) {
+                    sv[j] = (live && (!tail || tile_tok0 + j < it.kv_end)) ? sv[j] * p.scale_log2 : -INFINITY;  // (also drops what stale rows gave)
                     mx = fmaxf(mx, sv[j]);
                 }
-                mxs[ch * kRows + sm_row] = mx;
-                asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps: both column halves of a row are in
-                const float mn = fmaxf(m_run, fmaxf(mxs[sm_row], mxs[kRows + sm_row]));
+                const float mn = fmaxf(m_run, mx);
                 const float ms = (mn == -INFINITY) ? 0.f : mn;
                 const float a = fast_exp2(m_run - ms);
                 m_run = mn;
                 float sum = 0.f;
-                uint32_t pk[16];
+                uint8_t *prow = smem + kOffKV + b * kTileBytes + 8 * kPanelBytes + row * 128;  // panel 8 of the stage: free once the scores exist
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float p0 = fast_exp2(sv[2 * j] - ms), p1 = fast_exp2(sv[2 * j + 1] - ms);
-                    sum += p0 + p1;
-                    pk[j] = pack_bf16(p0, p1);
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float p0 = fast_exp2(sv[8 * c + 2 * j] - ms), p1 = fast_exp2(sv[8 * c + 2 * j + 1] - ms);
+                        sum += p0 + p1;
+                        pk[j] = pack_bf16(p0, p1);
+                    }
+                    *reinterpret_cast<uint4 *>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
                 l_run = l_run * a + sum;
-                uint4 *dst = reinterpret_cast<uint4 *>(smem + kOffP + sm_row * kPPitch + ch * 64);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                if (ch == 0) corr_s[sm_row] = a;
-                if (tr) t_softmax += clock64() - t0, t0 = clock64();
+                corr_s[b * kRows + row] = a;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_pready + b * 8);
             }
-            __syncthreads();  // (A) weights and correction factors of the tile are visible
-            if (tr) t_wait_a += clock64() - t0, t0 = clock64();
-
-            // ---- rescale, then O[16 rows, 256 latent columns] += P[16 x 64] . C[64 x 256] on mma.sync ----
-            const float a0 = corr_s[rb * 16 + g8], a1 = corr_s[rb * 16 + g8 + 8];
-            if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {
-#pragma unroll
-                for (int n = 0; n < kDv / 16; ++n) {
-                    o[n][0] *= a0;
-                    o[n][1] *= a0;
-                    o[n][2] *= a1;
-                    o[n][3] *= a1;
-                }
-            }
-            const bool more = tile + 1 < it.tile_end;  // the next tile belongs to the same item: its scores can be issued now
-            live = __all_sync(0xffffffffu, mbar_wait(bar_full + s_idx * 8, ph, abort_flag, p.error_flag, 24)) && live;  // (landed long ago: the scores came from it)
-            if (live) {
-                const int n_ks = tail ? min(4, (it.kv_end - tile_tok0 + 15) >> 4) : 4;
-                const uint32_t p_addr = p_smem + (rb * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * kPPitch + ((lane >> 4) << 4);
-                const int vr = (lane & 7) + (((lane >> 3) & 1) << 3);
-                const int v_csel = lane >> 4;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    // the elected thread looks between steps whether the next tile has landed and, if so, starts its scores
-                    if (tid == 0 && more && s_issued <= fill + 1 && mbar_try_wait(bar_full + ((fill + 1) % kStages) * 8, ((fill + 1) / kStages) & 1))
-                        issue_scores(fill + 1);
-                    __syncwarp();
-                    if (kk >= n_ks) continue;
-                    uint32_t pa[4];
-                    ldsm_x4(pa[0], pa[1], pa[2], pa[3], p_addr + kk * 32);
-                    uint32_t vmask0 = 0xffffffffu, vmask1 = 0xffffffffu;
-                    if (tail) {
-                        const int t0 = tile_tok0 + kk * 16 + 2 * q4;
-                        vmask0 = (t0 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 1 < it.kv_end ? 0xffff0000u : 0u);
-                        vmask1 = (t0 + 8 < it.kv_end ? 0x0000ffffu : 0u) | (t0 + 9 < it.kv_end ? 0xffff0000u : 0u);
-                    }
-                    const uint32_t row_addr = stage + (kk * 16 + vr) * 128;
-#pragma unroll
-                    for (int n2 = 0; n2 < kDv / 32; ++n2) {
-                        const int cg = ch * (kDv / 16) + 2 * n2 + v_csel;
-                        uint32_t b0, b1, b2, b3;
-                        ldsm_x4_t(b0, b1, b2, b3, row_addr + (cg >> 3) * kPanelBytes + (((cg & 7) ^ swz) << 4));
-                        b0 &= vmask0;
-                        b1 &= vmask1;
-                        b2 &= vmask0;
-                        b3 &= vmask1;
-                        mma_bf16(o[2 * n2], pa, b0, b1);
-                        mma_bf16(o[2 * n2 + 1], pa, b2, b3);
-                    }
-                }
-            }
-            if (tr) t_pv += clock64() - t0, t0 = clock64();
-            __syncthreads();  // (B) everybody is done with the weight tile and with this stage
-            if (tr) t_wait_b += clock64() - t0, t0 = clock64();
-            if (tid == 0) {
-                issue_next_copy();  // the tile two ahead, into the stage just freed (first: the copies must never wait for one another)
-                if (more && s_issued <= fill + 1) {  // the next tile had not landed while the steps ran: wait for it (bounded)
-                    if (mbar_wait(bar_full + ((fill + 1) % kStages) * 8, ((fill + 1) / kStages) & 1, abort_flag, p.error_flag, 25)) issue_scores(fill + 1);
-                }
-                if (tr) t_post += clock64() - t0;
-            }
+            lsum_s[(n_item & 1u) * kRows + row] = l_run;
+            mfin_s[(n_item & 1u) * kRows + row] = m_run;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_fin + (n_item & 1u) * 8);
         }
-
-        // ---- end of the item: row sums and maxima from the softmax threads, then the result ----
-        if (sm_warp) {
-            mxs[ch * kRows + sm_row] = l_run;
-            if (ch == 0) m_s[sm_row] = m_run;
+      } else if (warp == kMmaWarp) {
+        // ================= score MMAs: one lane issues, the warp follows item by item =================
+        uint32_t s_issued = 0;
+        for (int i = item_lo; i < item_hi; ++i) {
+            const MlaItem it = item_at(i);
+            __syncwarp();
+            asm volatile("bar.sync 1, 96;" ::: "memory");  // the softmax warps have put the item's query panels in place
+            if (lane == 0) {
+                for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++f) {
+                    const uint32_t b = f & 1u, ph = (f >> 1) & 1u;
+                    if (!mbar_wait_inl(bar_full + b * 8, ph, abort_flag, p.error_flag, 32)) continue;
+                    if (!mbar_wait_inl(bar_sfree + b * 8, ph ^ 1u, abort_flag, p.error_flag, 33)) continue;
+                    tc_fence_after();
+                    const uint64_t adesc = kDescHi | (uint64_t)((smem_base + kOffQ) >> 4);
+                    const uint64_t bdesc = kDescHi | (uint64_t)((smem_base + kOffKV + b * kTileBytes) >> 4);
+                    const uint32_t d = tmem_base + b * 64u;
+#pragma unroll
+                    for (int pn = 0; pn < kPanels; ++pn)
+#pragma unroll
+                        for (int k16 = 0; k16 < 4; ++k16) {
+                            const uint64_t off = (uint64_t)((pn * kPanelBytes + k16 * 32) >> 4);
+                            umma_bf16(d, adesc + off, bdesc + off, (pn | k16) ? 1u : 0u);
+                        }
+                    umma_commit(bar_sdone + b * 8);
+                    s_issued = f + 1;
+                }
+            }
+            __syncwarp();
         }
-        __syncthreads();
-        const int r0 = rb * 16 + g8, r1 = r0 + 8;
-        const float lt0 = mxs[r0] + mxs[kRows + r0], lt1 = mxs[r1] + mxs[kRows + r1];
-        const float m0 = m_s[r0], m1 = m_s[r1];
-        const float inv0 = lt0 > 0.f ? 1.f / lt0 : 0.f, inv1 = lt1 > 0.f ? 1.f / lt1 : 0.f;
-        if (live) {
-            if (it.partial_idx < 0) {
-                __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(p.out);
-                const int64_t base0 = ((int64_t)it.q_row * p.n_heads + it.head0 + r0) * kDv + ch * (kDv / 2) + 2 * q4;
-                const int64_t base1 = base0 + 8ll * kDv;
-#pragma unroll
-                for (int n = 0; n < kDv / 16; ++n) {
-                    *reinterpret_cast<uint32_t *>(out + base0 + n * 8) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
-                    *reinterpret_cast<uint32_t *>(out + base1 + n * 8) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
-                }
-                if (p.lse_out && ch == 0 && q4 == 0) {  // natural log
-                    p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r0] = lt0 > 0.f ? m0 * 0.6931471805599453f + logf(lt0) : -INFINITY;
-                    p.lse_out[(int64_t)it.q_row * p.n_heads + it.head0 + r1] = lt1 > 0.f ? m1 * 0.6931471805599453f + logf(lt1) : -INFINITY;
-                }
-            } else {
-                float *po = p.part_o + (int64_t)it.partial_idx * kRows * kDv;
-                const int64_t base0 = (int64_t)r0 * kDv + ch * (kDv / 2) + 2 * q4, base1 = base0 + 8ll * kDv;
-#pragma unroll
-                for (int n = 0; n < kDv / 16; ++n) {
-                    *reinterpret_cast<float2 *>(po + base0 + n * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
-                    *reinterpret_cast<float2 *>(po + base1 + n * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
-                }
-                if (ch == 0 && q4 == 0) {  // log2 domain
-                    p.part_lse[(int64_t)it.partial_idx * kRows + r0] = lt0 > 0.f ? m0 + log2f(lt0) : -INFINITY;
-                    p.part_lse[(int64_t)it.partial_idx * kRows + r1] = lt1 > 0.f ? m1 + log2f(lt1) : -INFINITY;
+        if (lane == 0 && *abort_flag) {  // a wait ran out: give the MMAs still in flight a bounded time before the tensor memory goes
+            for (uint32_t b = 0; b < 2; ++b) {
+                const uint32_t uses = (s_issued + 1 - b) / 2;
+                if (uses == 0) continue;
+                for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar_sdone + b * 8, (uses - 1) & 1); ++spin) {
                 }
             }
         }
-    }
-    if (tr && lane == 0 && (warp == 0 || warp == 2)) {
-        unsigned long long *w = p.trace + (size_t)blockIdx.x * kTraceWords + (warp == 0 ? 0 : 8);
-        w[0] = clock64() - t_all, w[1] = n_tiles, w[2] = t_wait_s, w[3] = t_softmax, w[4] = t_wait_a, w[5] = t_pv, w[6] = t_wait_b, w[7] = warp == 0 ? t_post : t_item;
-    }
-    // A wait ran out: give the copies and the MMAs still in flight a bounded time to finish before the CTA gives up its
-    // shared and tensor memory.
-    if (*abort_flag && tid == 0) {
-        for (uint32_t st = 0; st < kStages; ++st) {
-            const uint32_t uses = (c_fill + kStages - 1 - st) / kStages;
-            if (uses == 0) continue;
-            for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar_full + st * 8, (uses - 1) & 1); ++spin) {
+      } else if (lane == 0) {
+        // ================= tile copies =================
+        uint32_t c_fill = 0;
+        for (int i = item_lo; i < item_hi; ++i) {
+            const MlaItem it = item_at(i);
+            const char *kv = reinterpret_cast<const char *>(it.kv);
+            for (int tile = it.tile_begin; tile < it.tile_end; ++tile, ++f) {
+                const uint32_t b = f & 1u, ph = (f >> 1) & 1u;
+                if (!mbar_wait_inl(bar_stfree + b * 8, ph ^ 1u, abort_flag, p.error_flag, 31)) continue;
+                const int rows = min(T, (it.kv_end - tile * T + 15) & ~15);  // 16-token steps that hold visible tokens
+                mbar_expect_tx(bar_full + b * 8, kPanels * rows * 128);
+                const uint32_t dst = smem_base + kOffKV + b * kTileBytes;
+                const char *src = kv + (int64_t)tile * kTileBytes;
+                const int n_copy = ((int)blockIdx.x == p.debug_stall_cta && f == 0) ? kPanels - 1 : kPanels;  // test hook: the wait on this tile must run out
+#pragma unroll
+                for (int pn = 0; pn < kPanels; ++pn)
+                    if (pn < n_copy) bulk_g2s(dst + pn * kPanelBytes, src + pn * kPanelBytes, rows * 128, bar_full + b * 8);
+                c_fill = f + 1;
             }
         }
-        for (uint32_t b = 0; b < 2; ++b) {
-            const uint32_t uses = (s_issued + 1 - b) / 2;
-            if (uses == 0) continue;
-            for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar_sdone + b * 8, (uses - 1) & 1); ++spin) {
+        if (*abort_flag) {  // a wait ran out: give the copies still in flight a bounded time to land before the CTA gives up its shared memory
+            for (uint32_t b = 0; b < 2; ++b) {
+                const uint32_t uses = (c_fill + 1 - b) / 2;
+                if (uses == 0) continue;
+                for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(bar_full + b * 8, (uses - 1) & 1); ++spin) {
+                }
             }
         }
+      }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
 }
 
 // Merge of split units by their log-sum-exp weights: block (u, y) handles rows 4y..4y+3 of unit u; a thread owns four
@@ -778,7 +797,7 @@ int mla_configure_kernels() {
 
 int launch_mla_attention(const MlaLaunch &p, bool scores_on_tcgen05, void *stream) {
     if (scores_on_tcgen05)
-        return (int)launch_pdl(mla_attention_kernel_tc, dim3(p.n_ctas), dim3(kThreads), tc::kSmemBytes, static_cast<cudaStream_t>(stream), p);
+        return (int)launch_pdl(mla_attention_kernel_tc, dim3(p.n_ctas), dim3(tc::kThreadsWs), tc::kSmemBytes, static_cast<cudaStream_t>(stream), p);
     return (int)launch_pdl(mla_attention_kernel, dim3(p.n_ctas), dim3(kThreads), kSmemBytes, static_cast<cudaStream_t>(stream), p);
 }
 

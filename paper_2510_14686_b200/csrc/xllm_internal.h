@@ -185,7 +185,7 @@ struct MlaLaunch {
     const CombineDesc *comb_src;  // descriptors of the split units in mapped host memory ...
     CombineDesc *comb_dst;        // ... which the kernel copies here (device memory) for the combine kernel that follows
     int32_t n_comb;
-    unsigned long long *trace;    // optional per-CTA cycle counters (debug), may be null
+    int32_t debug_stall_cta;      // -1; else that CTA arms its first tile copy but leaves one panel out (timeout test)
     int32_t n_heads;
     float scale_log2;
     int32_t n_ctas;

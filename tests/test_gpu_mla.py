@@ -20,6 +20,13 @@ def binding():
     return b
 
 
+@pytest.fixture(params=["mma.sync", "tcgen05"], autouse=True)
+def kernel_choice(request, monkeypatch):
+    """Every test runs against both attention kernels: the library reads the choice when a context is created."""
+    monkeypatch.setenv("XLLM_MLA_KERNEL", request.param)
+    return request.param
+
+
 def mla_ctx(binding, n_heads, n_slots, max_seq_len, kv_lens, max_q_len=4):
     pages = sum(-(-(-(-int(t) // 64) * 64 * D * 2) // PAGE) for t in kv_lens) + 2
     return binding.Context(n_heads, 1, D, n_slots, max_seq_len, pages * PAGE, max_q_len=max_q_len, flags=binding.FLAG_MLA)
@@ -214,3 +221,32 @@ def test_bench_sized_batch_on_sampled_rows(binding, name):
         err = np.abs(got[rr][:, heads] - ref_o)
         assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (r, err.max(), err.mean())
         assert np.abs(got_lse[rr][:, heads] - ref_l).max() <= LSE_ABS
+
+
+def test_wait_runs_out_and_context_recovers(binding):
+    """One tile copy of one launch is left incomplete (a host-armed test hook): the bounded wait for it runs out, the launch
+    ends by itself (the tcgen05 kernel frees its tensor memory on the way), the error shows once, the context keeps working."""
+    import time
+
+    kv = [900, 70, 3000]
+    b = wl.mla_batch(2006, 128, kv)
+    with mla_ctx(binding, 128, len(kv), 4096, kv) as ctx:
+        slots = load(ctx, b)
+        good, lse = run(ctx, b, slots)
+        check(b, good, lse)
+        ctx.debug_inject_timeout(1)
+        from gpu_harness import dev_bits
+
+        q = dev_bits(b.q)
+        out = torch.zeros((q.shape[0], 128, wl.MLA_D_C), dtype=torch.int16, device="cuda")
+        t0 = time.monotonic()
+        ctx.mla_attention(slots, q, out, None, None, b.scale)
+        with pytest.raises(binding.XllmError) as ei:
+            ctx.sync_check()
+        took = time.monotonic() - t0
+        assert ei.value.status == binding.ERR_CUDA and "bounded device-side wait expired" in str(ei.value)
+        assert 1.0 < took < 20.0, took
+        ctx.sync_check()
+        for _ in range(2):
+            again, lse2 = run(ctx, b, slots)
+            assert np.array_equal(again, good) and np.array_equal(lse2, lse)

@@ -457,6 +457,12 @@ def run_mla(args):
     except Exception:
         tf_peak, hbm_peak, which = 1400.0, FALLBACK_HBM_GBS, "fallback"
     tf = flops / (attn_ms * 1e-3) / 1e12
+    traffic = None
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            traffic = json.load(f).get(f"mla_{name}")
+    except Exception:
+        pass
     print(json.dumps({"metric": METRIC, "value": int(kv.sum()) / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
                       "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
                       "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -464,7 +470,9 @@ def run_mla(args):
                                              f"contexts {int(kv.min())}..{int(kv.max())} tokens", "kv_copies_rotated": copies,
                                  "kv_bytes_per_step_per_gpu": kv_bytes, "l2": "inputs larger than L2 (rotating KV copies)"},
                       "roofline": {"bound": "tensor", "achieved": tf, "peak": tf_peak, "unit": "TFLOP/s", "frac": tf / tf_peak,
-                                   "traffic": None, "peak_source": which, "kernel": "mla_attention_kernel (mma.sync m16n8k16)",
+                                   "traffic": traffic, "peak_source": which,
+                                   "kernel": "mla_attention_kernel_tc (tcgen05 scores, mma.sync P.V)" if os.environ.get("XLLM_MLA_KERNEL") == "tcgen05"
+                                   else "mla_attention_kernel (mma.sync m16n8k16)",
                                    "kernel_ms": attn_ms, "combine_kernel_ms": comb_ms, "flops_per_launch": flops,
                                    "hbm_achieved_gbs": kv_bytes / (attn_ms * 1e-3) / 1e9,
                                    "hbm_frac": kv_bytes / (attn_ms * 1e-3) / 1e9 / hbm_peak},

@@ -586,7 +586,7 @@ xllm_status xllm_init(const xllm_config *cfg, xllm_ctx **out) {
     const int32_t groups = (G <= kMaxRows) ? (cfg->max_q_len + std::max(1, kMaxRows / G) - 1) / std::max(1, kMaxRows / G)
                                            : cfg->max_q_len * ((G + kMaxRows - 1) / kMaxRows);
     ctx->max_items = cfg->max_slots * cfg->n_kv_heads * groups + (1 + kPoolMaxPerCta) * ctx->sm_count + 1;
-    ctx->max_partials = 2 * ctx->sm_count + 2;
+    ctx->max_partials = 2 * ctx->sm_count + 2 + (mla ? 2 * (cfg->n_q_heads / kMlaRows) : 0);  // (MLA: one plan per head block, each with its own rounding)
     ctx->stage_bytes = std::max(align_up(sizeof(DevItem) * (size_t)ctx->max_items, 16) +
                                     align_up(sizeof(CombineDesc) * (size_t)ctx->max_partials, 16),
                                 align_up(sizeof(AppendDesc) * (size_t)cfg->max_slots, 16)) + 64;
@@ -1164,21 +1164,29 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     }
     const int32_t n_tok = (int32_t)tok_kv.size();
     const int32_t head_blocks = ctx->cfg.n_q_heads / kMlaRows;
-    int32_t n_units = 0, n_partials = 0;
+    // All head blocks of a token read the same latent tiles.  When the CTAs divide evenly, the work of ONE head block is
+    // planned over n_ctas / head_blocks CTAs and the other blocks get the same plan on the next groups of CTAs: the groups
+    // then walk the same tiles at the same time, and every fetch after the first one of a tile is an L2 hit.
+    const bool mirrored = head_blocks > 1 && ctx->sm_count % head_blocks == 0;
+    const int32_t reps = mirrored ? head_blocks : 1;
+    const int32_t plan_blocks = mirrored ? 1 : head_blocks, plan_ctas = ctx->sm_count / reps;
+    int32_t n_units = 0, n_partials_plan = 0;
     PlanTuning tune = ctx->tune;
     tune.pool_pct = 0;      // (no run-time pool in this kernel)
     tune.row_overhead = 0;  // every item carries the same 64 rows
-    if (plan_partition(n_tok, tok_kv.data(), nullptr, head_blocks, head_blocks, ctx->sm_count, tune, ctx->items, ctx->cta_begin,
-                       &n_units, &n_partials, &ctx->plan_scratch) != 0)
+    if (plan_partition(n_tok, tok_kv.data(), nullptr, plan_blocks, plan_blocks, plan_ctas, tune, ctx->items, ctx->cta_begin,
+                       &n_units, &n_partials_plan, &ctx->plan_scratch) != 0)
         return fail(ctx, XLLM_ERR_INVALID, std::string(who) + ": could not partition the work");
-    const int32_t n_items = (int32_t)ctx->items.size();
+    const int32_t n_items_plan = (int32_t)ctx->items.size();
+    const int32_t n_items = n_items_plan * reps, n_partials = n_partials_plan * reps;
     if (n_items > ctx->max_items || n_partials > ctx->max_partials)
         return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": work list exceeds the workspace sized at init");
     std::vector<CombineDesc> &combine = ctx->combine;
     combine.clear();
-    for (const xllm_work_item &it : ctx->items)
-        if (it.partial_idx >= 0 && it.partial_idx == it.part_first)  // first piece of a split unit
-            combine.push_back({it.part_first, it.n_parts, it.req, it.kv_head * kMlaRows, 1, kMlaRows});
+    for (int32_t rep = 0; rep < reps; ++rep)
+        for (const xllm_work_item &it : ctx->items)
+            if (it.partial_idx >= 0 && it.partial_idx == it.part_first)  // first piece of a split unit
+                combine.push_back({it.part_first + rep * n_partials_plan, it.n_parts, it.req, (it.kv_head + rep) * kMlaRows, 1, kMlaRows});
 
     int idx = -1;
     int e = acquire_stage(ctx, &idx);
@@ -1188,17 +1196,19 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
         return fail(ctx, XLLM_ERR_UNSUPPORTED, std::string(who) + ": staging buffer too small");
     char *h = ctx->h_stage[idx], *d = ctx->d_stage[idx];
     MlaItem *mi = reinterpret_cast<MlaItem *>(h);
-    for (int32_t i = 0; i < n_items; ++i) {
-        const xllm_work_item &w = ctx->items[(size_t)i];
-        const SlotRecord &s = ctx->xt->slot(slots[tok_req[(size_t)w.req]]);
-        mi[i].kv = s.base;
-        mi[i].q_row = w.req;  // query tokens are packed in request order: the planner's request index is the row
-        mi[i].head0 = w.kv_head * kMlaRows;
-        mi[i].tile_begin = w.tile_begin;
-        mi[i].tile_end = w.tile_end;
-        mi[i].kv_end = (int32_t)tok_kv[(size_t)w.req];
-        mi[i].partial_idx = w.partial_idx;
-    }
+    for (int32_t rep = 0; rep < reps; ++rep)
+        for (int32_t i = 0; i < n_items_plan; ++i) {
+            const xllm_work_item &w = ctx->items[(size_t)i];
+            const SlotRecord &s = ctx->xt->slot(slots[tok_req[(size_t)w.req]]);
+            MlaItem &m = mi[rep * n_items_plan + i];
+            m.kv = s.base;
+            m.q_row = w.req;  // query tokens are packed in request order: the planner's request index is the row
+            m.head0 = (w.kv_head + rep) * kMlaRows;
+            m.tile_begin = w.tile_begin;
+            m.tile_end = w.tile_end;
+            m.kv_end = (int32_t)tok_kv[(size_t)w.req];
+            m.partial_idx = w.partial_idx < 0 ? -1 : w.partial_idx + rep * n_partials_plan;
+        }
     if (!combine.empty()) std::memcpy(h + off_comb, combine.data(), sizeof(CombineDesc) * combine.size());
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -1216,7 +1226,9 @@ xllm_status xllm_mla_attention(xllm_ctx *ctx, int32_t n_req, const int32_t *slot
     ml.n_heads = ctx->cfg.n_q_heads;
     ml.scale_log2 = scale * 1.4426950408889634f;
     ml.n_ctas = ctx->sm_count;
-    std::memcpy(ml.cta_begin, ctx->cta_begin.data(), sizeof(int32_t) * (size_t)(ctx->sm_count + 1));
+    for (int32_t rep = 0; rep < reps; ++rep)  // CTA rep * plan_ctas + c runs the plan of CTA c on head block rep
+        for (int32_t c = 0; c < plan_ctas; ++c) ml.cta_begin[rep * plan_ctas + c] = rep * n_items_plan + ctx->cta_begin[(size_t)c];
+    ml.cta_begin[ctx->sm_count] = n_items;
     ml.debug_stall_cta = -1;
     if (ctx->inject_timeouts > 0) {
         --ctx->inject_timeouts;

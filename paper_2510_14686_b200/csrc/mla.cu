@@ -1,4 +1,6 @@
-// MLA (multi-head latent attention) decode / verification kernels of libxllm_attn.so (sm_100a), first version.
+// MLA (multi-head latent attention) decode / verification kernels of libxllm_attn.so (sm_100a): the whole contraction on
+// mma.sync (mla_attention_kernel, the default), and the same work with Q.K^T on tcgen05 + tensor memory
+// (mla_attention_kernel_tc, further down).
 //
 // The cache holds ONE vector per token, c = [latent (512 dims) | rotary key (64 dims)], shared by all heads; head h of
 // a query token carries q = [q_latent | q_rope] of the same 576 dims (weight-absorbed form).  Scores use all 576 dims,
@@ -15,8 +17,8 @@
 // shared memory, they do not fit registers), the two halves agree on row maxima through shared memory and exchange
 // their bf16 weights (the two warps of a row block synchronise with a 64-thread barrier of their own, so the four row
 // blocks drift apart and mix their load- and MMA-heavy phases), and for P.V the warp accumulates all 64 tokens into
-// latent columns 256 ch..256 ch+255 (128 fp32 registers per thread).  The contraction runs on mma.sync m16n8k16: with 128 heads per token this path is
-// as much tensor- as HBM-bound, and a tcgen05/TMEM version of the two contractions is the step after this one.
+// latent columns 256 ch..256 ch+255 (128 fp32 registers per thread).  Both contractions run on mma.sync m16n8k16
+// here: with 128 heads per token this path is as much tensor- as HBM-bound.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 

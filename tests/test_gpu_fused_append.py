@@ -113,10 +113,12 @@ def test_falls_back_to_two_launches_when_rows_exceed_one_group(binding):
     check_edge(out, lse, batch)
 
 
-def test_named_decode_workload_fused(binding):
+@pytest.mark.parametrize("name", ["decode", "verify", "longctx"])
+def test_named_workload_fused(binding, name):
+    """Full size, through the call the benchmark times: the step's new rows ride along with the attention launch."""
     import gpu_harness as gh
 
-    batch = wl.make_batch("decode")
+    batch = wl.make_batch(name)
     out, lse, launches = run_fused(binding, batch)
     assert launches == 0
     gh.assert_parity(out, lse, *gh.oracle_batch(batch))

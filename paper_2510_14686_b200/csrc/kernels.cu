@@ -348,6 +348,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
     uint32_t item_seq = 0;  // items started so far
     unsigned long long tr_tiles = 0, tr_wait_q = 0, tr_switch = 0, tr_wait_empty = 0, tr_first = 0, tr_epi = 0, tr_epi_main = 0;
 
+    const uint64_t kv_policy = l2_policy_evict_first();  // K/V tiles are read once: first in line for eviction from L2
     __syncthreads();          // barriers initialised
     grid_launch_dependents();  // the next kernel of the stream may start its own prologue
     grid_dependency_wait();    // from here on q, the KV ranges and the outputs may be touched
@@ -506,7 +507,7 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
                             const uint32_t dst = smem_base + C::kOffStages + hs * C::kHalfTile;
 #pragma unroll
                             for (int pn = 0; pn < C::kPanels; ++pn)
-                                bulk_g2s(dst + pn * kPanelBytes, src + (half * C::kPanels + pn) * kPanelBytes, bytes, bar_full + hs * 8);
+                                bulk_g2s_stream(dst + pn * kPanelBytes, src + (half * C::kPanels + pn) * kPanelBytes, bytes, bar_full + hs * 8, kv_policy);
                         }
                     }
                 }

@@ -432,6 +432,10 @@ def run_mla(args):
     st0 = ctx.get_stats().as_dict()
     sampler = ClockSampler(0)
     sampler.start()
+    t0, i = time.perf_counter(), 0
+    while sampler.proc and not sampler.lines and time.perf_counter() - t0 < 5.0:   # sampler start-up stays untimed
+        step(i)
+        i += 1
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     ev0.record()
@@ -526,6 +530,13 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     t_load0 = time.perf_counter()
+    # The sampler is a child process whose start-up (loading the management library, opening the device) takes a few
+    # hundred ms of host and driver time; the timed region of a short workload is ~10 ms.  Keep stepping, untimed,
+    # until its first sample has arrived, so that the start-up does not fall into the timed region.
+    i = 0
+    while rank == 0 and sampler.proc and not sampler.lines and time.perf_counter() - t_load0 < 5.0:
+        rep.step(i)
+        i += 1
     st0 = rep.ctx.get_stats()
     ms = timed(args.steps, rep.step)                                       # ---- the timed region ----
     st1 = rep.ctx.get_stats()
@@ -551,7 +562,8 @@ def run_ours(args):
 
     # keep the GPU under the same load until the clock sampler has seen it for a while
     i = 0
-    while rank == 0 and time.perf_counter() - t_load0 < 1.5:
+    t_load1 = time.perf_counter()
+    while rank == 0 and time.perf_counter() - t_load1 < 1.0:
         rep.step(i)
         i += 1
     torch.cuda.synchronize()

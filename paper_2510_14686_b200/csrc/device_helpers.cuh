@@ -104,6 +104,11 @@ __device__ __forceinline__ void bulk_g2s_stream(uint32_t dst, const void *src, u
                  "l"(src), "r"(bytes), "r"(bar), "l"(policy)
                  : "memory");
 }
+// Asks L2 to fetch a range.  A hint without effect on ordering or visibility: L2 is where every SM's writes land, so a
+// line requested early is still the current one when it is read later.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)

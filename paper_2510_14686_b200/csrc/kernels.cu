@@ -351,6 +351,15 @@ __device__ __forceinline__ void attention_body(const AttnHeader &p, const int it
     const uint64_t kv_policy = l2_policy_evict_first();  // K/V tiles are read once: first in line for eviction from L2
     __syncthreads();          // barriers initialised
     grid_launch_dependents();  // the next kernel of the stream may start its own prologue
+    // A CTA becomes resident while the previous kernel's last CTAs are still streaming, and idles until that kernel has
+    // drained.  In that time it asks L2 for the first tiles of its first item (whose record came with the parameters):
+    // the memory system stays busy through the kernel boundary and the rings then fill from L2.  Only a hint is issued
+    // here; every read of the data comes after the wait.
+    if (warp == kProducerWarp && lane == 0 && item_hi > item_lo && p.prefetch_tiles > 0) {
+        const char *kv0 = reinterpret_cast<const char *>(first_rec.kv);
+        const int n = min(first_rec.tile_end - first_rec.tile_begin, p.prefetch_tiles);
+        for (int t = 0; t < n; ++t) bulk_prefetch_l2(kv0 + (int64_t)(first_rec.tile_begin + t) * tile_block, 2 * C::kHalfTile);
+    }
     grid_dependency_wait();    // from here on q, the KV ranges and the outputs may be touched
     const unsigned long long g_go = TRACE ? globaltimer_ns() : 0ull;
     unsigned long long g_first = 0, g_last = 0;

@@ -902,7 +902,7 @@ xllm_status xllm_kv_append(xllm_ctx *ctx, int32_t n_req, const int32_t *slots, c
                       ctx->cfg.n_kv_heads, ctx->cfg.head_dim, stream);
     time_end(ctx, stream);
     if (e) return cuda_fail(ctx, "launching the append kernel", e);
-    ctx->st.kernel_launches += (n_desc + kAppendBatch - 1) / kAppendBatch;
+    ctx->st.kernel_launches += append_launch_count(n_desc);
     finish_launch(ctx, idx, stream);
     for (int32_t i = 0; i < n_req; ++i) {
         SlotRecord &s = ctx->xt->slot(slots[i]);

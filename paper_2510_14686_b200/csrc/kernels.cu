@@ -20,6 +20,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <type_traits>
 #include <utility>
 
 #include "xllm_internal.h"
@@ -969,7 +970,8 @@ __device__ __forceinline__ int64_t slot_chunk_offset(int64_t pos, int h, int whi
            (int64_t)which * (panels * kPanelBytes) + (c >> 3) * kPanelBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
 }
 
-__global__ void append_kernel(const __grid_constant__ AppendLaunch descs, const uint4 *__restrict__ k_new,
+template <class Launch>
+__global__ void append_kernel(const __grid_constant__ Launch descs, const uint4 *__restrict__ k_new,
                               const uint4 *__restrict__ v_new, int n_kv_heads, int D) {
     grid_launch_dependents();
     grid_dependency_wait();  // the previous kernel may still read the slots or write k_new / v_new
@@ -1103,14 +1105,21 @@ int launch_append(const AppendDesc *descs, int32_t n_req, int32_t max_new, const
     const int64_t per_req = 2ll * max_new * n_kv_heads * (head_dim / 8);  // chunks of the largest request
     const int threads = 256;
     const int64_t bx = std::min<int64_t>((per_req + threads - 1) / threads, 4096);
-    for (int32_t first = 0; first < n_req; first += kAppendBatch) {  // descriptors go by value: no trip to host memory
-        const int32_t n = std::min(kAppendBatch, n_req - first);
-        AppendLaunch al;
+    const auto launch = [&](auto &al, int32_t first, int32_t n) {  // descriptors go by value: no trip to host memory
         for (int32_t i = 0; i < n; ++i) al.d[i] = descs[first + i];
         dim3 grid((unsigned)bx, (unsigned)n);
-        const cudaError_t e = launch_pdl(append_kernel, grid, dim3(threads), 0, static_cast<cudaStream_t>(stream), al,
-                                         static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), (int)n_kv_heads,
-                                         (int)head_dim);
+        return launch_pdl(append_kernel<std::remove_reference_t<decltype(al)>>, grid, dim3(threads), 0, static_cast<cudaStream_t>(stream), al,
+                          static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new), (int)n_kv_heads, (int)head_dim);
+    };
+    if (n_req <= kAppendBatch) {
+        AppendLaunch al;
+        const cudaError_t e = launch(al, 0, n_req);
+        if (e != cudaSuccess) return (int)e;
+        return 0;
+    }
+    for (int32_t first = 0; first < n_req; first += kAppendBatchWide) {
+        AppendLaunchWide al;
+        const cudaError_t e = launch(al, first, std::min(kAppendBatchWide, n_req - first));
         if (e != cudaSuccess) return (int)e;
     }
     return 0;

@@ -121,6 +121,15 @@ constexpr int32_t kAppendBatch = 128;  // requests per append launch (their desc
 struct AppendLaunch {
     AppendDesc d[kAppendBatch];
 };
+// Calls with more requests than that take a wider record (12 KiB of parameters), so that a step of a few hundred
+// requests is still one append launch; small calls keep the short record.
+constexpr int32_t kAppendBatchWide = 512;
+struct AppendLaunchWide {
+    AppendDesc d[kAppendBatchWide];
+};
+inline int32_t append_launch_count(int32_t n_desc) {
+    return n_desc <= kAppendBatch ? (n_desc > 0 ? 1 : 0) : (n_desc + kAppendBatchWide - 1) / kAppendBatchWide;
+}
 
 // What every CTA of an attention launch needs: travels in the kernel parameters, or (graph mode) sits in host memory
 // mapped into the device and is fetched by each CTA when it starts.

@@ -166,3 +166,35 @@ def test_release_reuse_and_pressure_on_device(binding):
         assert np.array_equal(gk, k3)
         ctx.kv_release(b, 1)
         assert ctx.get_stats().pages_free == 3
+
+
+@pytest.mark.parametrize("n_req", [1, 128, 129, 512, 513, 1100])
+def test_append_of_many_requests_in_one_call_is_bit_exact(binding, n_req):
+    """One append call over n_req requests with 0..3 new rows each (the descriptor record of a launch holds 128 requests,
+    a wider one 512, larger calls take several launches): every slot gathers back exactly its own rows, in order."""
+    from gpu_harness import dev_bits
+
+    hkv, d = 2, 64
+    rng = np.random.default_rng(n_req)
+    n_new = rng.integers(0, 4, n_req).astype(np.int32)
+    n_new[0] = 3
+    rows = int(n_new.sum())
+    k = rng.integers(0, 1 << 16, (rows, hkv, d), dtype=np.uint16)
+    v = rng.integers(0, 1 << 16, (rows, hkv, d), dtype=np.uint16)
+    page = 2 << 20
+    with binding.Context(hkv * 4, hkv, d, n_req, 4096, n_req * page) as ctx:
+        slots = [ctx.kv_reserve() for _ in range(n_req)]
+        for s in slots:
+            ctx.kv_map_pages(s, 8)
+        before = ctx.get_stats().kernel_launches
+        ctx.kv_append(slots, n_new, dev_bits(k), dev_bits(v))
+        ctx.sync_check()
+        launches = ctx.get_stats().kernel_launches - before
+        assert launches == (1 if n_req <= 128 else -(-int((n_new > 0).sum()) // 512))
+        row0 = 0
+        for s, n in zip(slots, n_new):
+            assert ctx.kv_slot_info(s).kv_len == n
+            if n:
+                gk, gv = gather(ctx, s, 0, int(n), hkv, d)
+                assert np.array_equal(gk, k[row0:row0 + n]) and np.array_equal(gv, v[row0:row0 + n])
+            row0 += int(n)
